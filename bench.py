@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KV operator path on B200 (one JSON line on stdout).
+
+A step is one pass of the whole operator path over one batch of synthetic input, on the
+Llama-3-8B-shaped workload (32 layers, 8 KV heads, head_dim 128, block 16, bf16; pool of 32768
+blocks with a seeded-permuted free list), in its unaligned variant so that copy-on-write and the
+re-packing compose really copy:
+
+    import 8187-token context -> materialize to a transfer buffer -> import that buffer ->
+    fork to 16 agents -> one batched append of 16 x 512 tokens (each agent copies the shared
+    partial tail on write) -> compose(agent0, agent1) -> evict everything
+
+metric  = KV bytes moved (read + written) per second, whole job, inputs resident in HBM.
+e2e     = the same step with the step's inputs copied from pinned host memory and the
+          materialised transfer buffer copied back to the host inside the timed region.
+roofline= the copy kernel (the one kernel every operator's bytes go through): algorithmic bytes
+          per launch / its mean launch time from CUDA events recorded by the library on the
+          launching stream, against the measured HBM copy peak.
+cpu_baseline = the CPU oracle (plain single-threaded C) timed on a bounded sample of the same step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 8b|70b|tiny]
+N > 1 runs independent replicas (the path has no exchange step): launch with torch.distributed.run.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from workloads import configs, fill  # noqa: E402
+
+METRIC = "kv_bytes_moved_GBps"
+UNIT = "GB/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per algorithmic byte for the copy kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists)
+TRAFFIC_PER_ALGORITHMIC_BYTE = None
+
+
+def workload(name: str):
+    if name == "8b":
+        g = configs.LLAMA8B
+        return dict(name="llama3-8b-shaped KV, 8187-token context, 16 agents x 512 tokens, unaligned (COW)", g=g,
+                    seed=configs.SEED_BASE + 2, T=8187, agents=16, n_new=512)
+    if name == "70b":
+        g = configs.LLAMA70B
+        return dict(name="llama3-70b-shaped KV, 32763-token context, 8 agents x 1024 tokens, unaligned (COW)", g=g,
+                    seed=configs.SEED_BASE + 4, T=32763, agents=8, n_new=1024)
+    if name == "tiny":
+        g = configs.TINY
+        return dict(name="tiny pool, 507-token context, 4 agents x 64 tokens", g=g, seed=configs.SEED_BASE + 1,
+                    T=507, agents=4, n_new=64)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def class_tokens(g, T, agents, n_new):
+    """Tokens each operator class copies in one step (closed form of the step above)."""
+    r = T % g.block_size
+    la = T + n_new  # length of an agent after the append
+    rem = la % g.block_size
+    return {"materialize": T, "import": 2 * T, "append": agents * (n_new + r), "compose": (rem + la) if rem else 0}
+
+
+def step_ops(backend, root_buf, agent_bufs, T, agents, n_new, staging):
+    """One pass of the whole path on any backend with the KVPool method names. Returns #operators."""
+    st, root = backend.imp(root_buf, T)
+    assert st == 0, st
+    st, xfer = backend.materialize(root, 0, T, staging) if staging is not None else backend.materialize(root, 0, T)
+    assert st == 0, st
+    st, recv = backend.imp(xfer, T)
+    assert st == 0, st
+    st, kids = backend.fork(recv, agents)
+    assert st == 0, st
+    st, _ = backend.append(kids, [n_new] * agents, agent_bufs)
+    assert st == 0, st
+    st, merged = backend.compose(kids[:2], 0)
+    assert st == 0, st
+    st, _ = backend.evict([root, recv] + kids + [merged])
+    assert st == 0, st
+    return 7
+
+
+# ------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: str):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_rate(w, layers_sample: int, budget_s: float, max_steps: int):
+    """Times the CPU oracle, as it stands, on the same step restricted to `layers_sample` layers."""
+    from oracle import paged
+
+    g = w["g"]
+    paged.build()
+    o = paged.PagedOracle(layers_sample, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, g.n_blocks, g.max_ctx,
+                          g.max_blocks_per_ctx, configs.free_order(w["seed"], g.n_blocks))
+    per_layer = lambda n: 2 * n * g.row // 2
+    root = np.concatenate([fill.fill_np(w["seed"], 1, l * per_layer(w["T"]), per_layer(w["T"]))
+                           for l in range(layers_sample)]).view(np.uint8)
+    bufs = [np.concatenate([fill.fill_np(w["seed"], 2 + i, l * per_layer(w["n_new"]), per_layer(w["n_new"]))
+                            for l in range(layers_sample)]).view(np.uint8) for i in range(w["agents"])]
+
+    class B:  # adapter: the oracle's materialize allocates its own output
+        imp, fork, append, evict = o.imp, o.fork, o.append, o.evict
+        compose = staticmethod(lambda segs, fl: o.compose(segs, fl))
+        materialize = staticmethod(lambda c, a, b: o.materialize(c, a, b))
+
+    step_ops(B, root, bufs, w["T"], w["agents"], w["n_new"], None)  # warm-up (page faults of the pool)
+    rows0 = o.stats()["rows_copied"]
+    t0 = time.perf_counter()
+    steps = 0
+    while steps < max_steps and (steps == 0 or time.perf_counter() - t0 < budget_s):
+        step_ops(B, root, bufs, w["T"], w["agents"], w["n_new"], None)
+        steps += 1
+    dt = time.perf_counter() - t0
+    moved = 2 * (o.stats()["rows_copied"] - rows0) * g.row
+    return moved / dt / 1e9, steps, dt, 7 * steps / dt
+
+
+def reference_arm(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    layers = 2 if w["g"].n_layers > 2 else w["g"].n_layers
+    # `steps` timed passes, each a bounded sample of the workload (a subset of the layers)
+    gbps, steps, dt, ops_s = oracle_rate(w, layers, budget_s=1e9, max_steps=max(args.steps, 1))
+    cores = 1
+    sample = f"{layers} of {w['g'].n_layers} layers of the step, {steps} passes, single thread"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": 1, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": w["name"], "sample": sample},
+        "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "ops_per_s": ops_s,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "tiny"])
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST, 2 cp.async.bulk")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = workload(args.workload)
+    if args.impl == "reference":
+        reference_arm(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_10987_b200 import KVPool, binding
+
+    binding.load()  # fails loudly if the CUDA library is missing: there is no fallback
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    g, seed, T, agents, n_new = w["g"], w["seed"], w["T"], w["agents"], w["n_new"]
+    free_b, _total = torch.cuda.mem_get_info(dev)
+    n_blocks = g.n_blocks
+    need = lambda nb: g.n_layers * nb * 2 * g.run + 4 * T * g.bpt + (8 << 30)
+    while need(n_blocks) > free_b and n_blocks > 4096:
+        n_blocks //= 2  # recorded in config.n_blocks when the device lacks memory for the full pool
+    pool = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, n_blocks, g.max_ctx,
+                  g.max_blocks_per_ctx, free_order=configs.free_order(seed, n_blocks), device=local_rank)
+    pool.set_copy_engine(args.engine)
+    elems = lambda n: g.n_layers * 2 * n * g.row // 2
+    root_buf = fill.fill_torch(seed, 1, 0, elems(T), dev).view(torch.uint8)
+    agent_bufs = [fill.fill_torch(seed, 2 + i, 0, elems(n_new), dev).view(torch.uint8) for i in range(agents)]
+    staging = torch.empty(T * g.bpt, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def run(steps, fn):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    dev_step = lambda: step_ops(pool, root_buf, agent_bufs, T, agents, n_new, staging)
+
+    # ---- device-resident measurement
+    run(args.warmup, dev_step)
+    s0 = pool.stats()
+    pool.set_timing(True)
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    smi_id = vis.split(",")[local_rank].strip() if vis and local_rank < len(vis.split(",")) else str(local_rank)
+    sampler = ClockSampler(smi_id) if rank == 0 else None
+    ms = run(args.steps, dev_step)
+    clocks = sampler.stop() if sampler else None
+    pool.set_timing(False)
+    s1 = pool.stats()
+    assert pool.sync_status() == 0
+    moved_per_step = 2 * (s1["payload_bytes"] - s0["payload_bytes"]) / args.steps  # read + written
+    value = world * moved_per_step * args.steps / (ms * 1e-3) / 1e9
+    copy_launches = sum(s1["copy_launches"].values()) - sum(s0["copy_launches"].values())
+    meta_launches = s1["meta_launches"] - s0["meta_launches"]
+    copy_ms = sum(s1["copy_ms"].values()) - sum(s0["copy_ms"].values())
+    timed = sum(s1["timed_launches"].values()) - sum(s0["timed_launches"].values())
+    assert timed == copy_launches
+    achieved = moved_per_step * args.steps / (copy_ms * 1e-3) / 1e9
+
+    # ---- end to end: the step's inputs come from pinned host memory, the transfer buffer goes back
+    e2e = None
+    if not args.no_e2e:
+        h_root = torch.empty(T * g.bpt, dtype=torch.uint8).pin_memory()
+        h_agents = torch.empty(agents * n_new * g.bpt, dtype=torch.uint8).pin_memory()
+        h_out = torch.empty(T * g.bpt, dtype=torch.uint8).pin_memory()
+        h_root.copy_(root_buf)
+        h_agents.copy_(torch.cat(agent_bufs))
+        d_root = torch.empty_like(root_buf)
+        d_agents = torch.empty(agents * n_new * g.bpt, dtype=torch.uint8, device=dev)
+        views = [d_agents[i * n_new * g.bpt:(i + 1) * n_new * g.bpt] for i in range(agents)]
+
+        def e2e_step():
+            st, root = pool.import_host(h_root, T, d_root)  # H2D + scatter
+            assert st == 0, st
+            st = pool.materialize_host(root, 0, T, h_out, staging)  # gather + D2H
+            assert st == 0, st
+            st, recv = pool.imp(staging, T)
+            assert st == 0, st
+            st, kids = pool.fork(recv, agents)
+            assert st == 0, st
+            d_agents.copy_(h_agents, non_blocking=True)  # H2D of the continuation tokens
+            st, _ = pool.append(kids, [n_new] * agents, views)
+            assert st == 0, st
+            st, merged = pool.compose(kids[:2], 0)
+            assert st == 0, st
+            st, _ = pool.evict([root, recv] + kids + [merged])
+            assert st == 0, st
+
+        k_e2e = max(3, min(args.steps, 10))
+        run(1, e2e_step)
+        ms_e2e = run(k_e2e, e2e_step)
+        assert torch.equal(h_out, h_root), "end-to-end round trip changed the payload"
+        e2e = {"value": world * moved_per_step * k_e2e / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": (T + agents * n_new) * g.bpt, "d2h_bytes_per_step": T * g.bpt,
+               "ms_per_step": ms_e2e / k_e2e, "steps": k_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    per_launch_bytes = moved_per_step * args.steps / copy_launches
+    ct = class_tokens(g, T, agents, n_new)
+    assert 2 * sum(ct.values()) * g.bpt == moved_per_step, (ct, moved_per_step)
+    per_class = {}
+    for k, toks in ct.items():
+        dms = s1["copy_ms"][k] - s0["copy_ms"][k]
+        per_class[k] = (2 * toks * g.bpt * args.steps / (dms * 1e-3) / 1e9) if dms > 0 else None
+    roofline = {
+        "bound": "hbm", "kernel": "copy engine (aafkv::copy_vec_kernel / copy_bulk_kernel)", "achieved": achieved,
+        "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+        "frac_of_nominal_8TBps": achieved / 8000.0,
+        "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes if TRAFFIC_PER_ALGORITHMIC_BYTE else None),
+        "algorithmic_bytes_per_launch": per_launch_bytes, "launches": copy_launches,
+        "mean_launch_ms": copy_ms / copy_launches,
+        "per_class_GBps": per_class,
+    }
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        layers = 2 if g.n_layers > 2 else g.n_layers
+        gbps, steps_c, dt, _ = oracle_rate(w, layers, budget_s=12.0, max_steps=50)
+        cpu_baseline = {"value": gbps, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"{layers} of {g.n_layers} layers of the same step, {steps_c} passes in {dt:.1f} s, "
+                                  f"single thread of {len(os.sched_getaffinity(0))} available cores"}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": w["name"], "n_blocks": n_blocks, "pool_GiB": g.n_layers * n_blocks * 2 * g.run / 2**30,
+                   "l2_policy": "inputs_exceed_l2 (each operator streams >= 1 GiB)", "parallelism": "replicas only",
+                   "engine": args.engine, "moved_GB_per_step": moved_per_step / 1e9},
+        "ops_per_s": world * 7 * args.steps / (ms * 1e-3),
+        "gpu_launches": copy_launches + meta_launches,
+        "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

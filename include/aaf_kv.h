@@ -1,0 +1,223 @@
+/*
+ * aaf_kv.h -- C ABI of the B200 paged-KV operator library (libaafkv.so).
+ *
+ * The library implements the block-granular data movement behind the stateful KV
+ * operators of AAFLOW+ (arxiv 2607.10987): a paged KV pool whose contexts are block
+ * tables, with a device-resident free ring and reference-count table, and copy
+ * kernels for every path that moves KV bytes.
+ *
+ * Geometry and layouts (all sizes in bytes unless noted)
+ *   row   = n_kv_heads * head_dim * elt_bytes     one token, one layer, K or V
+ *   run   = block_size * row                      one block, one layer, K or V
+ *   bpt   = 2 * n_layers * row                    one token, all layers, K and V
+ *   pool  : device memory, layer l at pool_base + l * layer_stride_bytes, each layer
+ *           laid out [n_blocks][2 (K,V)][block_size][n_kv_heads][head_dim]; one block id
+ *           names the same slot range in every layer (Sec. 3.2: blocks b_j = (K_j, V_j,
+ *           layer, position range, device); Sec. 5.3: fixed-size block partitioning)
+ *   transfer buffer : dense [n_layers][2][n_tokens][n_kv_heads][head_dim], no header; the
+ *           metadata travels separately in an aaf_kv_xfer_desc (Sec. 5.4: raw tensor
+ *           buffers, metadata descriptors sent apart)
+ *   context: a block table (int32 block ids) plus a token count; token p lives in block
+ *           table[p / block_size], slot p % block_size (Sec. 5.3: the mapping
+ *           (state_id, block_id) -> (device, address))
+ *   refcount[b] = number of block-table entries that name block b (App. A.2, metadata
+ *           catalog: "refcount"); 0 <=> b is on the free ring
+ *
+ * Conventions the paper leaves open (stated so that results are reproducible):
+ *   allocation takes the oldest entries of the FIFO free ring in order; a block whose
+ *   refcount reaches 0 is pushed at the ring's tail, in (context, table position) order
+ *   of the evicting call; a new context gets the smallest free handle; no operator
+ *   writes a slot outside the tokens it stores; a failing call changes no state.
+ *
+ * Ownership: the caller owns ALL device memory (pool, workspace, transfer buffers) and
+ * keeps it valid while the pool object lives / until the stream has run the call.  The
+ * library allocates host memory only (the pool object, a pinned argument ring, events).
+ *
+ * Ordering: calls on one pool are applied in call order and must be issued to one stream
+ * (or the caller orders streams itself).  Data calls are asynchronous.  Not thread-safe
+ * per pool.  Pointers marked (device) must be device pointers, 16-byte aligned; row must
+ * be a multiple of 16.  Pointers marked (host) are ordinary host pointers read or
+ * written before the call returns.
+ *
+ * Errors: every call returns 0 (AAF_OK) or a negative aaf_status.  Everything the host
+ * can know is checked before anything is launched, so an error return means no state
+ * changed.  Conditions only the device can see (a corrupted ring or reference count, a
+ * bounded wait that gave up) never trap: they set a sticky status word that
+ * aaf_kv_sync_status returns and clears.
+ */
+#ifndef AAF_KV_H
+#define AAF_KV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AAF_KV_ABI_VERSION 1u
+
+typedef enum aaf_status {
+    AAF_OK = 0,
+    AAF_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, bad range, k < 1, duplicate ctx in a batch ... */
+    AAF_ERR_BAD_CTX = -2,       /* handle is not a live context                                             */
+    AAF_ERR_OOM_BLOCKS = -3,    /* not enough free blocks (exact: decided against the device's free count)  */
+    AAF_ERR_OOM_CTX = -4,       /* no free context handle                                                   */
+    AAF_ERR_TOO_LONG = -5,      /* result would exceed max_blocks_per_ctx                                   */
+    AAF_ERR_INCOMPAT = -6,      /* descriptor does not match the pool (Compat predicate, Sec. 3.2)          */
+    AAF_ERR_DST_TOO_SMALL = -7,
+    AAF_ERR_CUDA = -8,          /* a CUDA runtime call failed (no usable device, launch error ...)          */
+    AAF_ERR_CORRUPT = -9,       /* device found the ring / a reference count inconsistent                   */
+    AAF_ERR_TIMEOUT = -10,      /* a bounded device-side wait gave up                                       */
+    AAF_ERR_TOO_MANY = -11      /* batch larger than max_batch                                              */
+} aaf_status;
+
+typedef struct aaf_kv_pool aaf_kv_pool; /* opaque host object */
+typedef int32_t aaf_ctx_t;              /* context handle: slot index >= 0 */
+
+/* M and Theta of the KV state object S_KV = (M, Theta, B, Pi, Lambda, Gamma) (Sec. 3.2), the
+ * pool geometry, capacities and the caller-owned memory the pool lives in. */
+typedef struct aaf_kv_pool_desc {
+    uint32_t struct_size;        /* sizeof(aaf_kv_pool_desc)                                  */
+    uint32_t abi_version;        /* AAF_KV_ABI_VERSION                                        */
+    int32_t n_layers, n_kv_heads, head_dim, block_size, elt_bytes;
+    int32_t n_blocks;            /* blocks per layer in the pool                              */
+    int32_t max_ctx;             /* context handles 0 .. max_ctx-1                            */
+    int32_t max_blocks_per_ctx;  /* longest block table                                       */
+    int32_t max_batch;           /* largest n / m / k of a batched call (0 -> 1024)           */
+    int32_t device;              /* CUDA device ordinal that owns pool_base and workspace     */
+    void *pool_base;             /* (device) >= n_layers * layer_stride_bytes bytes           */
+    size_t layer_stride_bytes;   /* >= n_blocks * 2 * run, multiple of 16                     */
+    void *workspace;             /* (device) >= aaf_kv_pool_workspace_bytes(desc) bytes, 256-byte aligned */
+    size_t workspace_bytes;
+    const int32_t *free_order;   /* (host) permutation of [0, n_blocks) = initial ring, or NULL = identity */
+    uint64_t model_id;           /* M      : compared by the Compat predicate                 */
+    uint64_t config_hash;        /* Theta  : compared by the Compat predicate                 */
+} aaf_kv_pool_desc;
+
+/* Stand-in for the metadata descriptor that travels beside a transfer buffer (Sec. 5.4; Alg.
+ * "KV-Transfer": the descriptor is sent, then the raw buffers).  Host memory. */
+typedef struct aaf_kv_xfer_desc {
+    uint64_t model_id, config_hash;
+    int32_t n_layers, n_kv_heads, head_dim, elt_bytes;
+    int64_t pos_start;           /* Pi: position of the buffer's first token in its source context */
+    int64_t n_tokens;
+} aaf_kv_xfer_desc;
+
+#define AAF_COMPOSE_SHARE 0u     /* aligned segments share their full blocks by reference        */
+#define AAF_COMPOSE_COPY_ALL 1u  /* merge policy mu that forbids aliasing: everything is copied  */
+
+/* copy engines (aaf_kv_set_copy_engine) */
+#define AAF_ENGINE_AUTO 0        /* the library picks                                                     */
+#define AAF_ENGINE_VEC 1         /* 16-byte vector loads/stores through registers                         */
+#define AAF_ENGINE_BULK 2        /* cp.async.bulk global->shared->global with mbarrier completion         */
+
+/* operator classes that move payload (index into the per-class arrays of aaf_kv_stats) */
+#define AAF_OP_MATERIALIZE 0
+#define AAF_OP_IMPORT 1
+#define AAF_OP_APPEND 2
+#define AAF_OP_COMPOSE 3
+#define AAF_OP_CLASSES 4
+
+typedef struct aaf_kv_stats {
+    int64_t free_blocks, live_blocks;
+    int64_t peak_live_blocks;              /* Mem_KV = max_t sum ||KV_i(t)|| in blocks (Sec. 6.2)          */
+    int64_t live_ctx;
+    int64_t cow_count;                     /* partial tail blocks copied on write so far                   */
+    int64_t payload_bytes;                 /* bytes read (= bytes written) by the copy kernels so far      */
+    int64_t copy_launches[AAF_OP_CLASSES]; /* copy-kernel launches per operator class                      */
+    int64_t meta_launches;                 /* metadata (plan / fork / evict) kernel launches               */
+    double copy_ms[AAF_OP_CLASSES];        /* device time of the copy kernels per class, CUDA events on the
+                                              launching stream; only accumulated while timing is enabled   */
+    int64_t timed_launches[AAF_OP_CLASSES];
+} aaf_kv_stats;
+
+/* Workspace size for a geometry (pool_base / workspace / free_order fields are ignored).
+ * Returns 0 if the descriptor is invalid. */
+size_t aaf_kv_pool_workspace_bytes(const aaf_kv_pool_desc *desc);
+
+/* Pool creation: all reference counts 0, free ring = free_order, no context.  Writes the
+ * workspace on the device (synchronous).  The pool bytes themselves are not touched.
+ * Errors: INVALID_ARG (bad geometry, row not a multiple of 16, misaligned pointers, workspace
+ * too small, free_order not a permutation), CUDA. */
+int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out);
+int aaf_kv_pool_destroy(aaf_kv_pool *pool);
+
+/* materialize -- Alg. "KV-Transfer" (select the blocks of a position range, hand raw buffers to
+ * the transport), Sec. 5.4 (block granularity, prefix subsets).  Gathers tokens
+ * [tok_begin, tok_end) of ctx through its block table into the dense transfer buffer
+ * dst_dev (device, >= (tok_end - tok_begin) * bpt bytes): dst[l][kv][t - tok_begin] =
+ * pool[l][table[t / BS]][kv][t % BS].  Pure read of the pool.  out_desc (host, may be NULL)
+ * receives the descriptor.  Errors: BAD_CTX, INVALID_ARG (range, pointer), DST_TOO_SMALL. */
+int aaf_kv_materialize(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_dev,
+                       size_t dst_bytes, aaf_kv_xfer_desc *out_desc, void *stream);
+
+/* import -- Alg. "KV-Materialize" steps 4-6 (partition layer-wise K/V into blocks, register them)
+ * and Alg. "KV-Transfer" (register received blocks).  Scatters the desc->n_tokens tokens of
+ * src_dev (device) into ceil(n / BS) blocks taken from the free ring in order, each with
+ * refcount 1; *out_ctx (host) receives the new handle.  Only the slots of stored tokens are
+ * written.  Errors: INCOMPAT, INVALID_ARG, TOO_LONG, OOM_CTX, OOM_BLOCKS. */
+int aaf_kv_import(aaf_kv_pool *pool, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
+                  void *stream);
+
+/* fork -- Alg. "KV-Fork": k children alias the parent's blocks (table copied, refcount += 1 per
+ * entry per child); nothing is copied, no block allocated (Sec. 3.3).  out_children (host, k
+ * entries) receives the k smallest free handles in order.  Errors: BAD_CTX, INVALID_ARG, OOM_CTX,
+ * TOO_MANY. */
+int aaf_kv_fork(aaf_kv_pool *pool, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream);
+
+/* append -- Alg. "KV-Resume" (register continuation KV) with copy-on-write on divergence
+ * (Sec. 3.3; App. A.2).  For i < n: context ctxs[i] grows by n_new[i] tokens read from
+ * src_dev[i] (device, transfer layout [L][2][n_new[i]][H][D]).  If the context's partial tail
+ * block is shared, its valid rows are first copied into a fresh block and the old one is
+ * released.  The batch equals the for-loop over i; it is all-or-nothing.  ctxs, n_new, src_dev
+ * are host arrays.  Errors: BAD_CTX, INVALID_ARG (n_new < 1, duplicate ctx), TOO_LONG,
+ * OOM_BLOCKS, TOO_MANY. */
+int aaf_kv_append(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
+                  const void *const *src_dev, void *stream);
+
+/* compose -- Alg. "Restricted-KV-Merge", concatenation branch (Sec. 4.5): the new context is
+ * segs[0] || segs[1] || ... || segs[m-1], bytes verbatim.  A segment that starts on a block
+ * boundary shares its full blocks (and, if it is the last one, its partial tail) by reference;
+ * everything behind the first partial tail is re-packed into fresh blocks.  With
+ * AAF_COMPOSE_COPY_ALL nothing is shared.  Sources stay live; repeats allowed.  segs is a host
+ * array; *out_ctx (host).  Errors: BAD_CTX, INVALID_ARG, TOO_LONG, OOM_CTX, OOM_BLOCKS, TOO_MANY. */
+int aaf_kv_compose(aaf_kv_pool *pool, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
+                   void *stream);
+
+/* evict -- Alg. "KV-Evict", release step: every block-table entry of every listed context drops
+ * one reference; blocks that reach 0 return to the ring's tail in (context, table position)
+ * order; the handles become free.  Victim selection is the caller's policy.  ctxs is a host
+ * array.  Errors: BAD_CTX, INVALID_ARG (duplicate), TOO_MANY. */
+int aaf_kv_evict(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, void *stream);
+
+/* Host-buffer forms of the transfer pack / unpack (the device end of Sec. 5.4's transport when
+ * the peer is host memory).  staging_dev (device, >= n * bpt bytes) is caller-owned scratch.
+ * materialize_host gathers into staging_dev and copies it to dst_host; import_host copies
+ * src_host to staging_dev and scatters it.  Both enqueue on `stream`; host buffers must stay
+ * valid until the stream has run the call (use pinned memory for asynchronous copies). */
+int aaf_kv_materialize_host(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_host,
+                            size_t dst_bytes, void *staging_dev, size_t staging_bytes, aaf_kv_xfer_desc *out_desc,
+                            void *stream);
+int aaf_kv_import_host(aaf_kv_pool *pool, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
+                       size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream);
+
+/* Introspection (metadata catalog of App. A.2).  These synchronise the pool's stream. */
+int aaf_kv_ctx_len(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t *n_tokens);
+int aaf_kv_get_table(aaf_kv_pool *pool, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks);
+int aaf_kv_get_refcounts(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */);
+int aaf_kv_get_free_list(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */, int32_t *n_free);
+int aaf_kv_pool_stats(aaf_kv_pool *pool, aaf_kv_stats *out);
+/* Returns the sticky device status (AAF_OK, AAF_ERR_CORRUPT or AAF_ERR_TIMEOUT) and clears it. */
+int aaf_kv_sync_status(aaf_kv_pool *pool);
+
+/* Tuning and measurement knobs. */
+int aaf_kv_set_copy_engine(aaf_kv_pool *pool, int engine);  /* AAF_ENGINE_* */
+int aaf_kv_set_timing(aaf_kv_pool *pool, int enable);       /* bracket copy kernels with CUDA events */
+
+const char *aaf_kv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AAF_KV_H */

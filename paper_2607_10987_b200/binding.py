@@ -1,0 +1,317 @@
+"""ctypes binding of libaafkv.so: the same entry points as include/aaf_kv.h, argument
+marshalling only.  Every step of the path runs in the library's kernels; there is no Python
+or CPU fallback, and loading fails loudly if the shared library is missing.
+
+``KVPool`` is a convenience holder: it lets PyTorch allocate the pool, the workspace and
+transfer buffers (PyTorch is used for device memory and streams only) and forwards to the
+C entry points with the current stream.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaafkv.so")
+
+AAF_KV_ABI_VERSION = 1
+AAF_OK = 0
+AAF_ERR_INVALID_ARG, AAF_ERR_BAD_CTX, AAF_ERR_OOM_BLOCKS, AAF_ERR_OOM_CTX = -1, -2, -3, -4
+AAF_ERR_TOO_LONG, AAF_ERR_INCOMPAT, AAF_ERR_DST_TOO_SMALL, AAF_ERR_CUDA = -5, -6, -7, -8
+AAF_ERR_CORRUPT, AAF_ERR_TIMEOUT, AAF_ERR_TOO_MANY = -9, -10, -11
+AAF_COMPOSE_SHARE, AAF_COMPOSE_COPY_ALL = 0, 1
+AAF_ENGINE_AUTO, AAF_ENGINE_VEC, AAF_ENGINE_BULK = 0, 1, 2
+AAF_OP_MATERIALIZE, AAF_OP_IMPORT, AAF_OP_APPEND, AAF_OP_COMPOSE, AAF_OP_CLASSES = 0, 1, 2, 3, 4
+OP_NAMES = ("materialize", "import", "append", "compose")
+
+
+class aaf_kv_pool_desc(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("abi_version", C.c_uint32),
+        ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("block_size", C.c_int32),
+        ("elt_bytes", C.c_int32), ("n_blocks", C.c_int32), ("max_ctx", C.c_int32),
+        ("max_blocks_per_ctx", C.c_int32), ("max_batch", C.c_int32), ("device", C.c_int32),
+        ("pool_base", C.c_void_p), ("layer_stride_bytes", C.c_size_t),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("free_order", C.POINTER(C.c_int32)),
+        ("model_id", C.c_uint64), ("config_hash", C.c_uint64),
+    ]
+
+
+class aaf_kv_xfer_desc(C.Structure):
+    _fields_ = [
+        ("model_id", C.c_uint64), ("config_hash", C.c_uint64),
+        ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("elt_bytes", C.c_int32),
+        ("pos_start", C.c_int64), ("n_tokens", C.c_int64),
+    ]
+
+
+class aaf_kv_stats(C.Structure):
+    _fields_ = [
+        ("free_blocks", C.c_int64), ("live_blocks", C.c_int64), ("peak_live_blocks", C.c_int64),
+        ("live_ctx", C.c_int64), ("cow_count", C.c_int64), ("payload_bytes", C.c_int64),
+        ("copy_launches", C.c_int64 * AAF_OP_CLASSES), ("meta_launches", C.c_int64),
+        ("copy_ms", C.c_double * AAF_OP_CLASSES), ("timed_launches", C.c_int64 * AAF_OP_CLASSES),
+    ]
+
+
+# every symbol include/aaf_kv.h declares: name -> (restype, argtypes)
+_vp, _i32, _i64, _u32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_size_t
+_p32 = C.POINTER(C.c_int32)
+SYMBOLS = {
+    "aaf_kv_pool_workspace_bytes": (_sz, [C.POINTER(aaf_kv_pool_desc)]),
+    "aaf_kv_pool_create": (C.c_int, [C.POINTER(aaf_kv_pool_desc), C.POINTER(_vp)]),
+    "aaf_kv_pool_destroy": (C.c_int, [_vp]),
+    "aaf_kv_materialize": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
+    "aaf_kv_import": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _p32, _vp]),
+    "aaf_kv_fork": (C.c_int, [_vp, _i32, _i32, _p32, _vp]),
+    "aaf_kv_append": (C.c_int, [_vp, _i32, _p32, _p32, C.POINTER(_vp), _vp]),
+    "aaf_kv_compose": (C.c_int, [_vp, _i32, _p32, _u32, _p32, _vp]),
+    "aaf_kv_evict": (C.c_int, [_vp, _i32, _p32, _vp]),
+    "aaf_kv_materialize_host": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
+    "aaf_kv_import_host": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _p32, _vp]),
+    "aaf_kv_ctx_len": (C.c_int, [_vp, _i32, C.POINTER(_i64)]),
+    "aaf_kv_get_table": (C.c_int, [_vp, _i32, _p32, _i32, _p32]),
+    "aaf_kv_get_refcounts": (C.c_int, [_vp, _p32]),
+    "aaf_kv_get_free_list": (C.c_int, [_vp, _p32, _p32]),
+    "aaf_kv_pool_stats": (C.c_int, [_vp, C.POINTER(aaf_kv_stats)]),
+    "aaf_kv_sync_status": (C.c_int, [_vp]),
+    "aaf_kv_set_copy_engine": (C.c_int, [_vp, C.c_int]),
+    "aaf_kv_set_timing": (C.c_int, [_vp, C.c_int]),
+    "aaf_kv_strerror": (C.c_char_p, [C.c_int]),
+}
+
+_lib = None
+
+
+def load():
+    """Loads libaafkv.so (raises if it has not been built: there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_10987_b200._build` "
+                "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the KV operators."
+            )
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _fn(name):
+    return getattr(load(), name)
+
+
+# thin same-name wrappers ---------------------------------------------------------------------
+def aaf_kv_pool_workspace_bytes(desc): return _fn("aaf_kv_pool_workspace_bytes")(C.byref(desc))
+def aaf_kv_pool_create(desc, out): return _fn("aaf_kv_pool_create")(C.byref(desc), C.byref(out))
+def aaf_kv_pool_destroy(pool): return _fn("aaf_kv_pool_destroy")(pool)
+def aaf_kv_materialize(pool, ctx, t0, t1, dst, dst_bytes, out_desc, stream):
+    return _fn("aaf_kv_materialize")(pool, ctx, t0, t1, dst, dst_bytes, out_desc, stream)
+def aaf_kv_import(pool, src, desc, out_ctx, stream): return _fn("aaf_kv_import")(pool, src, desc, out_ctx, stream)
+def aaf_kv_fork(pool, parent, k, out_children, stream): return _fn("aaf_kv_fork")(pool, parent, k, out_children, stream)
+def aaf_kv_append(pool, n, ctxs, n_new, srcs, stream): return _fn("aaf_kv_append")(pool, n, ctxs, n_new, srcs, stream)
+def aaf_kv_compose(pool, m, segs, flags, out_ctx, stream): return _fn("aaf_kv_compose")(pool, m, segs, flags, out_ctx, stream)
+def aaf_kv_evict(pool, n, ctxs, stream): return _fn("aaf_kv_evict")(pool, n, ctxs, stream)
+def aaf_kv_materialize_host(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream):
+    return _fn("aaf_kv_materialize_host")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream)
+def aaf_kv_import_host(pool, src_host, desc, staging, staging_bytes, out_ctx, stream):
+    return _fn("aaf_kv_import_host")(pool, src_host, desc, staging, staging_bytes, out_ctx, stream)
+def aaf_kv_ctx_len(pool, ctx, out): return _fn("aaf_kv_ctx_len")(pool, ctx, out)
+def aaf_kv_get_table(pool, ctx, out, cap, n_blocks): return _fn("aaf_kv_get_table")(pool, ctx, out, cap, n_blocks)
+def aaf_kv_get_refcounts(pool, out): return _fn("aaf_kv_get_refcounts")(pool, out)
+def aaf_kv_get_free_list(pool, out, n_free): return _fn("aaf_kv_get_free_list")(pool, out, n_free)
+def aaf_kv_pool_stats(pool, out): return _fn("aaf_kv_pool_stats")(pool, out)
+def aaf_kv_sync_status(pool): return _fn("aaf_kv_sync_status")(pool)
+def aaf_kv_set_copy_engine(pool, engine): return _fn("aaf_kv_set_copy_engine")(pool, engine)
+def aaf_kv_set_timing(pool, enable): return _fn("aaf_kv_set_timing")(pool, enable)
+def aaf_kv_strerror(status): return _fn("aaf_kv_strerror")(status).decode()
+
+
+def make_desc(n_layers, n_kv_heads, head_dim, block_size, elt_bytes, n_blocks, max_ctx, max_blocks_per_ctx,
+              max_batch=0, device=0, model_id=0, config_hash=0) -> aaf_kv_pool_desc:
+    d = aaf_kv_pool_desc()
+    d.struct_size = C.sizeof(aaf_kv_pool_desc)
+    d.abi_version = AAF_KV_ABI_VERSION
+    d.n_layers, d.n_kv_heads, d.head_dim, d.block_size, d.elt_bytes = n_layers, n_kv_heads, head_dim, block_size, elt_bytes
+    d.n_blocks, d.max_ctx, d.max_blocks_per_ctx, d.max_batch, d.device = n_blocks, max_ctx, max_blocks_per_ctx, max_batch, device
+    d.model_id, d.config_hash = model_id, config_hash
+    return d
+
+
+class KVPool:
+    """Holds the torch-allocated memory of one pool and forwards to the C ABI.
+
+    Methods return (status, result); nothing is computed on the Python side.
+    """
+
+    def __init__(self, n_layers, n_kv_heads, head_dim, block_size, elt_bytes, n_blocks, max_ctx,
+                 max_blocks_per_ctx, free_order=None, max_batch=0, device=0, model_id=1, config_hash=1,
+                 pool_tensor=None):
+        import numpy as np
+        import torch
+
+        self.torch = torch
+        self.device = torch.device("cuda", device)
+        self.L, self.H, self.D, self.BS, self.E, self.NB = n_layers, n_kv_heads, head_dim, block_size, elt_bytes, n_blocks
+        self.max_ctx, self.max_blk = max_ctx, max_blocks_per_ctx
+        self.row = n_kv_heads * head_dim * elt_bytes
+        self.run = block_size * self.row
+        self.bpt = 2 * n_layers * self.row
+        self.layer_stride = n_blocks * 2 * self.run
+        d = make_desc(n_layers, n_kv_heads, head_dim, block_size, elt_bytes, n_blocks, max_ctx, max_blocks_per_ctx,
+                      max_batch, device, model_id, config_hash)
+        ws_bytes = aaf_kv_pool_workspace_bytes(d)
+        if ws_bytes == 0:
+            raise ValueError("invalid pool geometry")
+        if pool_tensor is None:
+            pool_tensor = torch.empty(n_layers * self.layer_stride, dtype=torch.uint8, device=self.device)
+        assert pool_tensor.numel() * pool_tensor.element_size() >= n_layers * self.layer_stride
+        self.pool = pool_tensor
+        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
+        d.pool_base, d.layer_stride_bytes = self.pool.data_ptr(), self.layer_stride
+        d.workspace, d.workspace_bytes = self.workspace.data_ptr(), ws_bytes
+        self._fo = None
+        if free_order is not None:
+            self._fo = np.ascontiguousarray(np.asarray(free_order, dtype=np.int32))
+            d.free_order = self._fo.ctypes.data_as(_p32)
+        self.desc = d
+        self.h = C.c_void_p()
+        st = aaf_kv_pool_create(d, self.h)
+        if st != AAF_OK:
+            raise RuntimeError(f"aaf_kv_pool_create failed: {aaf_kv_strerror(st)}")
+
+    # ------------------------------------------------------------------ helpers
+    def _stream(self):
+        return C.c_void_p(self.torch.cuda.current_stream(self.device).cuda_stream)
+
+    def xfer_desc(self, n_tokens, pos_start=0) -> aaf_kv_xfer_desc:
+        x = aaf_kv_xfer_desc()
+        x.model_id, x.config_hash = self.desc.model_id, self.desc.config_hash
+        x.n_layers, x.n_kv_heads, x.head_dim, x.elt_bytes = self.L, self.H, self.D, self.E
+        x.pos_start, x.n_tokens = pos_start, n_tokens
+        return x
+
+    def close(self):
+        if getattr(self, "h", None) and self.h.value:
+            aaf_kv_pool_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ operators
+    def materialize(self, ctx, t0, t1, out=None):
+        n = max(t1 - t0, 0)
+        if out is None:
+            out = self.torch.empty(max(n * self.bpt, 16), dtype=self.torch.uint8, device=self.device)
+        xd = aaf_kv_xfer_desc()
+        st = aaf_kv_materialize(self.h, ctx, t0, t1, out.data_ptr(), out.numel() * out.element_size(), C.byref(xd),
+                                self._stream())
+        return st, (out if st == AAF_OK else None)
+
+    def imp(self, buf, n, desc=None):
+        xd = desc if desc is not None else self.xfer_desc(n)
+        out = C.c_int32(-1)
+        st = aaf_kv_import(self.h, buf.data_ptr(), C.byref(xd), C.byref(out), self._stream())
+        return st, (out.value if st == AAF_OK else None)
+
+    def fork(self, parent, k):
+        out = (C.c_int32 * max(k, 1))()
+        st = aaf_kv_fork(self.h, parent, k, out, self._stream())
+        return st, (list(out[:k]) if st == AAF_OK else None)
+
+    def append(self, ctxs, n_new, bufs):
+        n = len(ctxs)
+        a = (C.c_int32 * max(n, 1))(*ctxs)
+        b = (C.c_int32 * max(n, 1))(*n_new)
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in bufs])
+        return aaf_kv_append(self.h, n, a, b, ptrs, self._stream()), None
+
+    def compose(self, segs, flags=0):
+        m = len(segs)
+        a = (C.c_int32 * max(m, 1))(*segs)
+        out = C.c_int32(-1)
+        st = aaf_kv_compose(self.h, m, a, flags, C.byref(out), self._stream())
+        return st, (out.value if st == AAF_OK else None)
+
+    def evict(self, ctxs):
+        n = len(ctxs)
+        a = (C.c_int32 * max(n, 1))(*ctxs)
+        return aaf_kv_evict(self.h, n, a, self._stream()), None
+
+    def materialize_host(self, ctx, t0, t1, dst_host, staging):
+        return aaf_kv_materialize_host(self.h, ctx, t0, t1, dst_host.data_ptr(),
+                                       dst_host.numel() * dst_host.element_size(), staging.data_ptr(),
+                                       staging.numel() * staging.element_size(), None, self._stream())
+
+    def import_host(self, src_host, n, staging):
+        xd = self.xfer_desc(n)
+        out = C.c_int32(-1)
+        st = aaf_kv_import_host(self.h, src_host.data_ptr(), C.byref(xd), staging.data_ptr(),
+                                staging.numel() * staging.element_size(), C.byref(out), self._stream())
+        return st, (out.value if st == AAF_OK else None)
+
+    # ------------------------------------------------------------------ introspection
+    def ctx_len(self, ctx):
+        v = C.c_int64(-1)
+        return v.value if aaf_kv_ctx_len(self.h, ctx, C.byref(v)) == AAF_OK else None
+
+    def table(self, ctx):
+        import numpy as np
+
+        out = np.empty(self.max_blk, dtype=np.int32)
+        nb = C.c_int32(0)
+        st = aaf_kv_get_table(self.h, ctx, out.ctypes.data_as(_p32), self.max_blk, C.byref(nb))
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        return out[: nb.value].copy()
+
+    def refcounts(self):
+        import numpy as np
+
+        out = np.empty(self.NB, dtype=np.int32)
+        st = aaf_kv_get_refcounts(self.h, out.ctypes.data_as(_p32))
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        return out
+
+    def free_list(self):
+        import numpy as np
+
+        out = np.empty(self.NB, dtype=np.int32)
+        nf = C.c_int32(0)
+        st = aaf_kv_get_free_list(self.h, out.ctypes.data_as(_p32), C.byref(nf))
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        return out[: nf.value].copy()
+
+    def live_ctxs(self):
+        return [c for c in range(self.max_ctx) if self.ctx_len(c) is not None]
+
+    def stats(self) -> dict:
+        s = aaf_kv_stats()
+        st = aaf_kv_pool_stats(self.h, C.byref(s))
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        d = {k: getattr(s, k) for k in ("free_blocks", "live_blocks", "peak_live_blocks", "live_ctx", "cow_count",
+                                        "payload_bytes", "meta_launches")}
+        d["copy_launches"] = dict(zip(OP_NAMES, list(s.copy_launches)))
+        d["copy_ms"] = dict(zip(OP_NAMES, list(s.copy_ms)))
+        d["timed_launches"] = dict(zip(OP_NAMES, list(s.timed_launches)))
+        return d
+
+    def sync_status(self):
+        return aaf_kv_sync_status(self.h)
+
+    def set_copy_engine(self, engine):
+        return aaf_kv_set_copy_engine(self.h, engine)
+
+    def set_timing(self, enable):
+        return aaf_kv_set_timing(self.h, 1 if enable else 0)

@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libaafkv.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "aaf_kv.h"
+
+namespace aafkv {
+
+// One contiguous copy, described once for all (layer, K/V) planes:
+//   plane (l, kv):  src + l * src_sl + kv * src_skv  ->  dst + l * dst_sl + kv * dst_skv,  nbytes bytes.
+// For a pool operand the strides are (layer_stride, run); for an n-token transfer buffer they are
+// (2 * n * row, n * row).  nbytes is a multiple of row (hence of 16); 0 marks an unused slot.
+struct __align__(16) Piece {
+    const char *src;
+    char *dst;
+    long long src_sl, src_skv;
+    long long dst_sl, dst_skv;
+    unsigned int nbytes;
+    unsigned int pad[3];
+};
+static_assert(sizeof(Piece) == 64, "Piece must be 64 bytes");
+
+// Device-resident control block at the start of the workspace.
+struct DevCtl {
+    unsigned long long head;   // ring counters: free = tail - head
+    unsigned long long tail;
+    int status;                // sticky: first AAF_ERR_CORRUPT / AAF_ERR_TIMEOUT seen by a kernel
+    int status_detail;
+    unsigned long long payload_bytes;  // bytes moved by copy kernels (one direction)
+    unsigned long long cow_count;
+    long long peak_live;
+    unsigned long long probe_need;     // dry-run result of the append planner
+    unsigned long long pad[9];
+};
+static_assert(sizeof(DevCtl) == 128, "DevCtl layout");
+
+struct Geom {
+    int L, H, D, BS, E, NB, max_ctx, max_blk;
+    long long row, run, layer_stride;
+    char *pool;
+};
+
+// Device views of the workspace.
+struct DevState {
+    DevCtl *ctl;
+    int *refcount;   // [NB]
+    int *ring;       // [NB]
+    int *last_pos;   // [NB] scratch of evict, -1 when idle
+    int *tables;     // [max_ctx][max_blk]
+    Piece *pieces;   // [max_pieces]
+    int *scratch;    // [3 * max_batch] per-batch scratch of the append planner
+};
+
+// ---- per-call argument records (written by the host into pinned memory, read by planners)
+struct AppendEntry {      // 32 bytes
+    const char *src;      // device payload [L][2][n_new][row]
+    long long T;          // tokens before the append
+    int ctx;
+    int n_new;
+    int piece_off;        // first piece slot of this entry (slot 0 = COW piece)
+    int pad;
+};
+struct ComposeSeg {       // 48 bytes
+    long long T;          // tokens of the segment
+    long long off;        // token offset of the segment in the result
+    int ctx;
+    int mode;             // 0 = share (aligned), 1 = copy
+    int share_tail;       // share mode: 1 = partial tail shared by reference (last segment)
+    int work_off;         // first flattened work item of the segment
+    int fresh_start;      // rank (from ring head) of the first fresh block the segment allocates
+    int piece_off;        // first piece slot of the segment
+    int dst_tbl_start;    // share mode: first result-table index written
+    int pad;
+};
+struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
+    int n;
+    int total;
+};
+
+// ---- launchers (each returns cudaGetLastError() of its launches)
+cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
+                                    cudaStream_t st);
+cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
+                               cudaStream_t st);
+cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, int nblk, int k, const int *children_dev,
+                        cudaStream_t st);
+cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
+                               int total_slots, int max_batch, int dry_run, cudaStream_t st);
+cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
+                                int total_fresh, int total_slots, int out_ctx, cudaStream_t st);
+cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
+                         cudaStream_t st);
+cudaError_t launch_copy(int engine, const Geom &g, const DevState &s, int n_slots, int plane0, int n_planes,
+                        int sm_count, cudaStream_t st);
+cudaError_t copy_engine_init(int device);
+
+}  // namespace aafkv

@@ -1,0 +1,264 @@
+// Copy engines of libaafkv.so: every byte a KV operator moves goes through one of the two
+// kernels below.  Both consume the same piece list (see Piece): a launch covers
+// n_slots pieces x n_planes (layer, K/V) planes, split into chunks of at most `chunk` bytes.
+//
+// The path is pure streaming (each byte is read once and written once, nothing is reused), so
+// the bound is HBM bandwidth: what matters is enough independent 16-byte accesses in flight per
+// SM, fully coalesced, and a grid that is a multiple of the SM count.
+//
+//   VEC  : 256 threads per CTA, each thread keeps UNROLL 16-byte streaming loads in flight and
+//          then stores them; grid-stride over chunks with a persistent grid.
+//   BULK : one elected thread per CTA drives a ring of shared-memory stages with
+//          cp.async.bulk (global -> shared, completion on an mbarrier) and
+//          cp.async.bulk (shared -> global, bulk async-group); no registers touch the data.
+//          Every wait is bounded; on expiry the kernel records AAF_ERR_TIMEOUT and leaves.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#include "aafkv_internal.h"
+
+namespace aafkv {
+
+// ------------------------------------------------------------------------------------------
+// unit decomposition shared by both engines: unit u -> (chunk c, piece p, plane q), plane-major
+// so that neighbouring CTAs stream neighbouring addresses of the dense side.
+struct Unit {
+    const char *src;
+    char *dst;
+    unsigned nbytes;  // 0 = nothing to do
+};
+
+__device__ __forceinline__ Unit decode_unit(const Piece *__restrict__ pieces, long long u, int n_slots, int plane0,
+                                            int cpp, unsigned chunk) {
+    const int c = (int)(u % cpp);
+    const long long t = u / cpp;
+    const int p = (int)(t % n_slots);
+    const int q = plane0 + (int)(t / n_slots);
+    const uint4 *pw = reinterpret_cast<const uint4 *>(pieces + p);
+    const uint4 w0 = __ldg(pw), w1 = __ldg(pw + 1), w2 = __ldg(pw + 2), w3 = __ldg(pw + 3);
+    Piece pc;
+    reinterpret_cast<uint4 *>(&pc)[0] = w0;
+    reinterpret_cast<uint4 *>(&pc)[1] = w1;
+    reinterpret_cast<uint4 *>(&pc)[2] = w2;
+    reinterpret_cast<uint4 *>(&pc)[3] = w3;
+    Unit r;
+    const unsigned off = (unsigned)c * chunk;
+    if (off >= pc.nbytes) {
+        r.src = nullptr; r.dst = nullptr; r.nbytes = 0;
+        return r;
+    }
+    const long long l = q >> 1, kv = q & 1;
+    r.src = pc.src + l * pc.src_sl + kv * pc.src_skv + off;
+    r.dst = pc.dst + l * pc.dst_sl + kv * pc.dst_skv + off;
+    r.nbytes = min(chunk, pc.nbytes - off);
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------
+// VEC engine
+constexpr int VEC_THREADS = 256;
+
+template <int UNROLL>
+__global__ void __launch_bounds__(VEC_THREADS) copy_vec_kernel(const Piece *__restrict__ pieces, int n_slots,
+                                                               int plane0, int n_planes, int cpp) {
+    constexpr unsigned CHUNK = VEC_THREADS * UNROLL * 16;
+    const long long total = (long long)n_slots * n_planes * cpp;
+    for (long long u = blockIdx.x; u < total; u += gridDim.x) {
+        const Unit un = decode_unit(pieces, u, n_slots, plane0, cpp, CHUNK);
+        if (un.nbytes == 0) continue;
+        const uint4 *__restrict__ s4 = reinterpret_cast<const uint4 *>(un.src);
+        uint4 *__restrict__ d4 = reinterpret_cast<uint4 *>(un.dst);
+        const unsigned nvec = un.nbytes >> 4;
+        uint4 v[UNROLL];
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const unsigned i = threadIdx.x + k * VEC_THREADS;
+            if (i < nvec) v[k] = __ldcs(s4 + i);
+        }
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const unsigned i = threadIdx.x + k * VEC_THREADS;
+            if (i < nvec) __stcs(d4 + i, v[k]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// BULK engine
+constexpr int BULK_MAX_STAGES = 8;
+constexpr long long BULK_WAIT_CYCLES = 1ll << 32;  // about two seconds of SM clock
+
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait: false if the phase did not complete within BULK_WAIT_CYCLES
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > BULK_WAIT_CYCLES) return false;
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_g2s(unsigned smem_dst, const void *gsrc, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_dst),
+                 "l"(gsrc), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *gdst, unsigned smem_src, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__ pieces, int n_slots, int plane0,
+                                                       int n_planes, int cpp, unsigned chunk, int stages,
+                                                       DevCtl *ctl) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bars[BULK_MAX_STAGES];
+    if (threadIdx.x != 0) return;
+
+    const long long total = (long long)n_slots * n_planes * cpp;
+    const unsigned smem0 = smem_u32(smem);
+    for (int s = 0; s < stages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+    char *dstq[BULK_MAX_STAGES];
+    unsigned nbq[BULK_MAX_STAGES];
+    long long u_next = blockIdx.x;  // next unit to look at for loading
+    int k_load = 0;                 // units whose load has been issued
+    int k_store = 0;                // units whose store has been issued
+    bool timed_out = false;
+
+    // finds the next non-empty unit and issues its load into stage k_load % stages
+    auto issue_load = [&]() -> bool {
+        while (u_next < total) {
+            const Unit un = decode_unit(pieces, u_next, n_slots, plane0, cpp, chunk);
+            u_next += gridDim.x;
+            if (un.nbytes == 0) continue;
+            const int s = k_load % stages;
+            const unsigned bar = smem_u32(&bars[s]);
+            mbar_expect_tx(bar, un.nbytes);
+            bulk_g2s(smem0 + (unsigned)s * chunk, un.src, un.nbytes, bar);
+            dstq[s] = un.dst;
+            nbq[s] = un.nbytes;
+            ++k_load;
+            return true;
+        }
+        return false;
+    };
+
+    for (int i = 0; i < stages - 1; ++i)
+        if (!issue_load()) break;
+
+    while (k_store < k_load) {
+        const int s = k_store % stages;
+        if (!mbar_wait_bounded(smem_u32(&bars[s]), (unsigned)(k_store / stages) & 1u)) {
+            timed_out = true;
+            break;
+        }
+        bulk_s2g(dstq[s], smem0 + (unsigned)s * chunk, nbq[s]);
+        bulk_commit();
+        ++k_store;
+        // the stage of the store before this one is the next load target: wait until that store has
+        // finished reading shared memory (the store just issued may stay pending)
+        bulk_wait_read_1();
+        issue_load();
+    }
+    if (timed_out) {
+        atomicCAS(&ctl->status, 0, (int)AAF_ERR_TIMEOUT);
+        // loads still in flight target this CTA's shared memory: give each one bounded wait before leaving
+        for (int k = k_store + 1; k < k_load; ++k)
+            mbar_wait_bounded(smem_u32(&bars[k % stages]), (unsigned)(k / stages) & 1u);
+    }
+    bulk_wait_all();
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+
+static int g_bulk_chunk = 16384;
+static int g_bulk_stages = 4;
+static int g_bulk_ctas_per_sm = 3;
+static int g_vec_unroll = 4;
+static int g_vec_ctas_per_sm = 8;
+static int g_auto_engine = AAF_ENGINE_VEC;
+
+static int env_int(const char *name, int dflt, int lo, int hi) {
+    const char *v = getenv(name);
+    if (!v || !*v) return dflt;
+    long x = strtol(v, nullptr, 10);
+    if (x < lo || x > hi) return dflt;
+    return (int)x;
+}
+
+// Reads the tuning knobs (environment, for experiments) and opts the bulk kernel in to the shared
+// memory it needs.  Called once per pool creation with the pool's device current.
+cudaError_t copy_engine_init(int device) {
+    (void)device;
+    g_bulk_chunk = env_int("AAFKV_BULK_CHUNK", g_bulk_chunk, 1024, 65536) & ~15;
+    g_bulk_stages = env_int("AAFKV_BULK_STAGES", g_bulk_stages, 2, BULK_MAX_STAGES);
+    g_bulk_ctas_per_sm = env_int("AAFKV_BULK_CTAS", g_bulk_ctas_per_sm, 1, 16);
+    g_vec_unroll = env_int("AAFKV_VEC_UNROLL", g_vec_unroll, 1, 8);
+    g_vec_ctas_per_sm = env_int("AAFKV_VEC_CTAS", g_vec_ctas_per_sm, 1, 8);
+    g_auto_engine = env_int("AAFKV_ENGINE", g_auto_engine, 1, 2);
+    while ((long long)g_bulk_chunk * g_bulk_stages > 220 * 1024) --g_bulk_stages;
+    return cudaFuncSetAttribute(copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                g_bulk_chunk * g_bulk_stages);
+}
+
+template <int UNROLL>
+static void launch_vec(const DevState &s, int n_slots, int plane0, int n_planes, long long run, int sm_count,
+                       cudaStream_t st) {
+    constexpr long long CHUNK = (long long)VEC_THREADS * UNROLL * 16;
+    const int cpp = (int)((run + CHUNK - 1) / CHUNK);
+    const long long total = (long long)n_slots * n_planes * cpp;
+    const long long cap = (long long)sm_count * g_vec_ctas_per_sm;
+    const int grid = (int)(total < cap ? total : cap);
+    copy_vec_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp);
+}
+
+cudaError_t launch_copy(int engine, const Geom &g, const DevState &s, int n_slots, int plane0, int n_planes,
+                        int sm_count, cudaStream_t st) {
+    if (n_slots <= 0 || n_planes <= 0) return cudaSuccess;
+    if (engine == AAF_ENGINE_AUTO) engine = g_auto_engine;
+    if (engine == AAF_ENGINE_BULK) {
+        const int cpp = (int)((g.run + g_bulk_chunk - 1) / g_bulk_chunk);
+        const long long total = (long long)n_slots * n_planes * cpp;
+        const long long cap = (long long)sm_count * g_bulk_ctas_per_sm;
+        const int grid = (int)(total < cap ? total : cap);
+        copy_bulk_kernel<<<grid, 32, (size_t)g_bulk_chunk * g_bulk_stages, st>>>(
+            s.pieces, n_slots, plane0, n_planes, cpp, (unsigned)g_bulk_chunk, g_bulk_stages, s.ctl);
+    } else {
+        switch (g_vec_unroll) {
+            case 1: launch_vec<1>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            case 2: launch_vec<2>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            case 8: launch_vec<8>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            default: launch_vec<4>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+        }
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace aafkv

@@ -1,0 +1,453 @@
+// Metadata kernels of libaafkv.so: the device-resident block allocator (FIFO free ring),
+// the reference-count table and the block tables, plus the planners that turn an operator
+// into a piece list for the copy engines.
+//
+// Determinism: which block a table entry gets, and where a freed block lands on the ring, must
+// be a function of the call sequence alone.  So a batch makes ONE reservation on the ring
+// (head advances once, by the batch's total need) and every entry finds its blocks at a
+// prefix-sum offset from the old head; reference counts are updated with atomics whose order
+// cannot change the result; frees are compacted in flattened (context, table position) order
+// by a block-wide prefix scan.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "aafkv_internal.h"
+
+namespace aafkv {
+
+constexpr int PLAN_THREADS = 1024;
+
+__device__ __forceinline__ void set_status(DevCtl *ctl, int code, int detail) {
+    if (atomicCAS(&ctl->status, 0, code) == 0) ctl->status_detail = detail;
+}
+__device__ __forceinline__ void note_alloc(DevCtl *ctl, const Geom &g, unsigned long long new_head,
+                                           unsigned long long tail) {
+    const long long live = (long long)g.NB - (long long)(tail - new_head);
+    if (live > ctl->peak_live) ctl->peak_live = live;
+}
+__device__ __forceinline__ int ring_at(const int *ring, unsigned long long pos, int NB) {
+    return ring[pos % (unsigned long long)NB];
+}
+__device__ __forceinline__ Piece make_piece(const char *src, long long ssl, long long sskv, char *dst, long long dsl,
+                                            long long dskv, unsigned nbytes) {
+    Piece p;
+    p.src = src; p.dst = dst;
+    p.src_sl = ssl; p.src_skv = sskv;
+    p.dst_sl = dsl; p.dst_skv = dskv;
+    p.nbytes = nbytes;
+    p.pad[0] = p.pad[1] = p.pad[2] = 0;
+    return p;
+}
+__device__ __forceinline__ char *pool_slot(const Geom &g, int b, long long slot) {
+    return g.pool + (long long)b * 2 * g.run + slot * g.row;
+}
+// takes a fresh block for exclusive use; a block on the ring must be unreferenced
+__device__ __forceinline__ void claim_block(const DevState &s, int b, int NB) {
+    if (b < 0 || b >= NB) {
+        set_status(s.ctl, AAF_ERR_CORRUPT, 1);
+        return;
+    }
+    if (s.refcount[b] != 0) set_status(s.ctl, AAF_ERR_CORRUPT, 2);
+    s.refcount[b] = 1;
+}
+
+// CTA-wide exclusive prefix sum of one int per thread (warp shuffles + one shared array).
+// Returns the exclusive prefix of `v`; *total receives the CTA's sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int *total) {
+    __shared__ int warp_sums[32];
+    __shared__ int block_total;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    __syncthreads();  // protects warp_sums / block_total of a previous call
+    if (lane == 31) warp_sums[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        int w = lane < nw ? warp_sums[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += t;
+        }
+        warp_sums[lane] = wi - w;  // exclusive prefix of the warp sums
+        if (lane == 31) block_total = wi;
+    }
+    __syncthreads();
+    *total = block_total;
+    return warp_sums[wid] + incl - v;
+}
+
+// ------------------------------------------------------------------------------------------
+// materialize: one piece per block of the token range
+__global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState s, int ctx, long long t0,
+                                                               long long t1, char *dst) {
+    const long long j0 = t0 / g.BS, j1 = (t1 - 1) / g.BS;
+    const long long n = t1 - t0;
+    const int *table = s.tables + (long long)ctx * g.max_blk;
+    for (long long j = j0 + blockIdx.x * blockDim.x + threadIdx.x; j <= j1; j += (long long)gridDim.x * blockDim.x) {
+        const long long lo = max(t0, j * g.BS), hi = min(t1, (j + 1) * g.BS);
+        const int b = table[j];
+        s.pieces[j - j0] = make_piece(pool_slot(g, b, lo - j * g.BS), g.layer_stride, g.run, dst + (lo - t0) * g.row,
+                                      2 * n * g.row, n * g.row, (unsigned)((hi - lo) * g.row));
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(n * 2 * g.L * g.row));
+}
+
+// ------------------------------------------------------------------------------------------
+// import: reserve ceil(n / BS) ring entries in order, write the table, one piece per block
+__global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevState s, int ctx, long long n,
+                                                                   const char *src) {
+    const int nblk = (int)((n + g.BS - 1) / g.BS);
+    const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
+    const bool ok = (tail - head0) >= (unsigned long long)nblk;
+    int *table = s.tables + (long long)ctx * g.max_blk;
+    for (int j = threadIdx.x; j < nblk; j += blockDim.x) {
+        if (!ok) {
+            s.pieces[j].nbytes = 0;
+            continue;
+        }
+        const int b = ring_at(s.ring, head0 + j, g.NB);
+        claim_block(s, b, g.NB);
+        table[j] = b;
+        const long long lo = (long long)j * g.BS, hi = min(n, lo + g.BS);
+        s.pieces[j] = make_piece(src + lo * g.row, 2 * n * g.row, n * g.row, pool_slot(g, b, 0), g.layer_stride, g.run,
+                                 (unsigned)((hi - lo) * g.row));
+    }
+    __syncthreads();  // every thread has read head0 before it moves
+    if (threadIdx.x == 0) {
+        if (!ok) {
+            set_status(s.ctl, AAF_ERR_CORRUPT, 3);
+        } else {
+            s.ctl->head = head0 + nblk;
+            note_alloc(s.ctl, g, head0 + nblk, tail);
+            s.ctl->payload_bytes += (unsigned long long)(n * 2 * g.L * g.row);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// fork: k table copies, refcount += k per parent entry
+__global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int parent, int nblk, int k,
+                                                   const int *__restrict__ children) {
+    const int *pt = s.tables + (long long)parent * g.max_blk;
+    const long long total = (long long)nblk * k;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int q = (int)(e / nblk), j = (int)(e % nblk);
+        const int b = pt[j];
+        s.tables[(long long)children[q] * g.max_blk + j] = b;
+        if (q == 0) atomicAdd(&s.refcount[b], k);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// append (+ copy-on-write)
+//
+// Sequential meaning of a batch: entry i copies its partial tail block iff the block is still
+// shared when the loop reaches i.  Among the batch entries whose partial tail is the same block b,
+// the one with rank q (q-th in array order) therefore copies iff q < refcount_before[b] - 1; the
+// entry that finds the count at 1 appends in place.  It writes only slots >= r while the copiers
+// read slots < r, so the batch's copies have no ordering hazard.
+//
+// scratch layout (ints): tailb[n] | need[n] | alloc_off[n]
+__global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevState s,
+                                                                   const AppendEntry *__restrict__ ent, int n,
+                                                                   int total_slots, int max_batch, int dry_run) {
+    int *tailb = s.scratch;
+    int *need = s.scratch + max_batch;
+    int *alloc_off = s.scratch + 2 * max_batch;
+    __shared__ int sh_total_need;
+    const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
+
+    // phase 1: the partial tail block of every entry (-1 if the context ends on a block boundary)
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const long long T = ent[i].T;
+        const int r = (int)(T % g.BS);
+        tailb[i] = r > 0 ? s.tables[(long long)ent[i].ctx * g.max_blk + (T - 1) / g.BS] : -1;
+    }
+    __syncthreads();
+    // phase 2: copy-on-write decision and block need of every entry
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const long long T = ent[i].T;
+        const int b = tailb[i];
+        int cow = 0;
+        if (b >= 0) {
+            int rank = 0;
+            for (int i2 = 0; i2 < i; ++i2) rank += (tailb[i2] == b);
+            cow = rank < s.refcount[b] - 1;
+        }
+        const int fresh = (int)((T + ent[i].n_new + g.BS - 1) / g.BS - (T + g.BS - 1) / g.BS);
+        need[i] = (cow << 30) | (cow + fresh);  // bit 30 remembers the decision
+    }
+    __syncthreads();
+    // phase 3: exclusive scan of the needs -> offset of each entry's blocks from the old ring head
+    int carry = 0;
+    for (int base = 0; base < n; base += blockDim.x) {
+        const int i = base + threadIdx.x;
+        const int v = i < n ? (need[i] & 0x3fffffff) : 0;
+        int tot;
+        const int ex = block_exclusive_scan(v, &tot);
+        if (i < n) alloc_off[i] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) sh_total_need = carry;
+    __syncthreads();
+    const int total_need = sh_total_need;
+    if (dry_run) {
+        if (threadIdx.x == 0) s.ctl->probe_need = (unsigned long long)total_need;
+        return;
+    }
+    const bool ok = (tail - head0) >= (unsigned long long)total_need;
+
+    // phase 4: one thread per piece slot.  Slot piece_off[i] is entry i's copy-on-write piece, the
+    // slots behind it are the blocks its new tokens touch, in table order.
+    for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) {
+        if (!ok) {
+            s.pieces[sl].nbytes = 0;
+            continue;
+        }
+        int lo = 0, hi = n - 1;  // last entry whose piece_off <= sl
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (ent[mid].piece_off <= sl) lo = mid; else hi = mid - 1;
+        }
+        const int i = lo;
+        const AppendEntry e = ent[i];
+        const long long T = e.T;
+        const int r = (int)(T % g.BS);
+        const int cow = (need[i] >> 30) & 1;
+        const unsigned long long first = head0 + (unsigned long long)alloc_off[i];
+        int *table = s.tables + (long long)e.ctx * g.max_blk;
+        const long long nblk_T = (T + g.BS - 1) / g.BS;
+        const int w = sl - e.piece_off;
+        if (w == 0) {
+            if (cow) {
+                const int old = tailb[i];
+                const int nb = ring_at(s.ring, first, g.NB);
+                claim_block(s, nb, g.NB);
+                if (atomicSub(&s.refcount[old], 1) <= 1) set_status(s.ctl, AAF_ERR_CORRUPT, 4);
+                table[nblk_T - 1] = nb;
+                s.pieces[sl] = make_piece(pool_slot(g, old, 0), g.layer_stride, g.run, pool_slot(g, nb, 0),
+                                          g.layer_stride, g.run, (unsigned)(r * g.row));
+                atomicAdd(&s.ctl->cow_count, 1ull);
+                atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(r * g.row * 2 * g.L));
+            } else {
+                s.pieces[sl].nbytes = 0;
+            }
+            continue;
+        }
+        const long long jpos = T / g.BS + (w - 1);  // table position of the touched block
+        int b;
+        if (jpos >= nblk_T) {  // a fresh continuation block
+            b = ring_at(s.ring, first + cow + (unsigned long long)(jpos - nblk_T), g.NB);
+            claim_block(s, b, g.NB);
+            table[jpos] = b;
+        } else {  // the partial tail: the copy if there is one, else written in place
+            b = cow ? ring_at(s.ring, first, g.NB) : tailb[i];
+        }
+        const long long tlo = max(T, jpos * g.BS), thi = min(T + e.n_new, (jpos + 1) * g.BS);
+        s.pieces[sl] = make_piece(e.src + (tlo - T) * g.row, 2ll * e.n_new * g.row, (long long)e.n_new * g.row,
+                                  pool_slot(g, b, tlo - jpos * g.BS), g.layer_stride, g.run,
+                                  (unsigned)((thi - tlo) * g.row));
+        atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((thi - tlo) * g.row * 2 * g.L));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (!ok) {
+            set_status(s.ctl, AAF_ERR_CORRUPT, 5);
+        } else {
+            s.ctl->head = head0 + total_need;
+            note_alloc(s.ctl, g, head0 + total_need, tail);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// compose: flattened over the work items of all segments (host supplies the prefix sums of the
+// lengths, which it knows; block ids come from the ring at rank offsets from the old head).
+//   share segment : item w < full -> share entry w; item w == full -> the partial tail (shared by
+//                   reference if it ends the result, else re-packed into a fresh block through the
+//                   segment's single piece slot)
+//   copy segment  : item w -> destination block nblk(off)-(off%BS>0) + w, which receives tokens
+//                   from at most two source blocks (two piece slots per item)
+__global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
+                                                                    const ComposeSeg *__restrict__ segs, int m,
+                                                                    int total_work, int total_fresh, int total_slots,
+                                                                    int out_ctx) {
+    const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
+    const bool ok = (tail - head0) >= (unsigned long long)total_fresh;
+    int *out = s.tables + (long long)out_ctx * g.max_blk;
+    if (!ok) {
+        for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) s.pieces[sl].nbytes = 0;
+    }
+    for (int it = threadIdx.x; ok && it < total_work; it += blockDim.x) {
+        int lo = 0, hi = m - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (segs[mid].work_off <= it) lo = mid; else hi = mid - 1;
+        }
+        const ComposeSeg sg = segs[lo];
+        const int w = it - sg.work_off;
+        const int *st = s.tables + (long long)sg.ctx * g.max_blk;
+        if (sg.mode == 0) {
+            const long long full = sg.T / g.BS;
+            const int rem = (int)(sg.T % g.BS);
+            if (w < full || sg.share_tail) {
+                const int b = st[w];
+                out[sg.dst_tbl_start + w] = b;
+                atomicAdd(&s.refcount[b], 1);
+            } else {  // w == full, rem > 0, not the last segment: re-pack the tail (the segment's one piece slot)
+                const int nb = ring_at(s.ring, head0 + (unsigned long long)sg.fresh_start, g.NB);
+                claim_block(s, nb, g.NB);
+                out[sg.dst_tbl_start + w] = nb;
+                s.pieces[sg.piece_off] = make_piece(pool_slot(g, st[full], 0), g.layer_stride, g.run,
+                                                    pool_slot(g, nb, 0), g.layer_stride, g.run,
+                                                    (unsigned)(rem * g.row));
+                atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(rem * g.row * 2 * g.L));
+            }
+        } else {
+            const long long nblk_off = (sg.off + g.BS - 1) / g.BS;
+            const long long d = sg.off / g.BS + w;  // destination table position
+            const int db = ring_at(s.ring, head0 + (unsigned long long)(sg.fresh_start + (d - nblk_off)), g.NB);
+            if (d >= nblk_off) {  // allocated by this segment
+                claim_block(s, db, g.NB);
+                out[d] = db;
+            }
+            const long long lo_t = max(sg.off, d * g.BS), hi_t = min(sg.off + sg.T, (d + 1) * g.BS);
+            const long long s_lo = lo_t - sg.off, s_hi = hi_t - sg.off;  // source token range
+            const long long sb0 = s_lo / g.BS;
+            const long long a_hi = min(s_hi, (sb0 + 1) * g.BS);
+            Piece *pp = s.pieces + sg.piece_off + 2 * w;
+            pp[0] = make_piece(pool_slot(g, st[sb0], s_lo - sb0 * g.BS), g.layer_stride, g.run,
+                               pool_slot(g, db, lo_t - d * g.BS), g.layer_stride, g.run,
+                               (unsigned)((a_hi - s_lo) * g.row));
+            if (a_hi < s_hi) {
+                pp[1] = make_piece(pool_slot(g, st[sb0 + 1], 0), g.layer_stride, g.run,
+                                   pool_slot(g, db, lo_t - d * g.BS + (a_hi - s_lo)), g.layer_stride, g.run,
+                                   (unsigned)((s_hi - a_hi) * g.row));
+            } else {
+                pp[1].nbytes = 0;
+            }
+            atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((s_hi - s_lo) * g.row * 2 * g.L));
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (!ok) {
+            set_status(s.ctl, AAF_ERR_CORRUPT, 6);
+        } else {
+            s.ctl->head = head0 + total_fresh;
+            note_alloc(s.ctl, g, head0 + total_fresh, tail);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// evict
+//   kernel A (grid)  : every flattened entry drops one reference and records the largest
+//                      flattened position at which its block occurs in the batch.
+//   kernel B (1 CTA) : a block is freed by the entry at its LAST occurrence iff its count is now 0
+//                      (that is where the sequential loop would have freed it); freed ids are
+//                      compacted in flattened order by a prefix scan and pushed at the ring's tail.
+__device__ __forceinline__ int evict_entry_block(const Geom &g, const DevState &s, const int *ctx, const int *ent_off,
+                                                 int n, int e) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (ent_off[mid] <= e) lo = mid; else hi = mid - 1;
+    }
+    return s.tables[(long long)ctx[lo] * g.max_blk + (e - ent_off[lo])];
+}
+
+__global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a) {
+    const int n = a->n, total = a->total;
+    const int *ctx = reinterpret_cast<const int *>(a + 1);
+    const int *ent_off = ctx + n;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int b = evict_entry_block(g, s, ctx, ent_off, n, e);
+        if (atomicSub(&s.refcount[b], 1) <= 0) set_status(s.ctl, AAF_ERR_CORRUPT, 7);
+        atomicMax(&s.last_pos[b], e);
+    }
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
+                                                                  const EvictArgs *__restrict__ a) {
+    const int n = a->n, total = a->total;
+    const int *ctx = reinterpret_cast<const int *>(a + 1);
+    const int *ent_off = ctx + n;
+    const unsigned long long tail0 = s.ctl->tail;
+    int carry = 0;
+    for (int base = 0; base < total; base += blockDim.x) {
+        const int e = base + threadIdx.x;
+        int b = -1, flag = 0;
+        if (e < total) {
+            b = evict_entry_block(g, s, ctx, ent_off, n, e);
+            flag = (s.refcount[b] == 0 && s.last_pos[b] == e);
+        }
+        int tot;
+        const int ex = block_exclusive_scan(flag, &tot);
+        if (flag) s.ring[(tail0 + (unsigned long long)(carry + ex)) % (unsigned long long)g.NB] = b;
+        carry += tot;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < total; e += blockDim.x)
+        s.last_pos[evict_entry_block(g, s, ctx, ent_off, n, e)] = -1;
+    if (threadIdx.x == 0) {
+        if (tail0 + carry - s.ctl->head > (unsigned long long)g.NB) set_status(s.ctl, AAF_ERR_CORRUPT, 8);
+        s.ctl->tail = tail0 + carry;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// launchers
+
+static int grid_for(long long items, int threads, int cap) {
+    long long gsz = (items + threads - 1) / threads;
+    if (gsz < 1) gsz = 1;
+    if (gsz > cap) gsz = cap;
+    return (int)gsz;
+}
+
+cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
+                                    cudaStream_t st) {
+    const long long nb = (t1 - 1) / g.BS - t0 / g.BS + 1;
+    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst);
+    return cudaGetLastError();
+}
+cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
+                               cudaStream_t st) {
+    plan_import_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, ctx, n, src);
+    return cudaGetLastError();
+}
+cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, int nblk, int k, const int *children_dev,
+                        cudaStream_t st) {
+    fork_kernel<<<grid_for((long long)nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, nblk, k, children_dev);
+    return cudaGetLastError();
+}
+cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
+                               int total_slots, int max_batch, int dry_run, cudaStream_t st) {
+    plan_append_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, entries_dev, n, total_slots, max_batch, dry_run);
+    return cudaGetLastError();
+}
+cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
+                                int total_fresh, int total_slots, int out_ctx, cudaStream_t st) {
+    plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, m, total_work, total_fresh, total_slots, out_ctx);
+    return cudaGetLastError();
+}
+cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
+                         cudaStream_t st) {
+    (void)n;
+    evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev);
+    return cudaGetLastError();
+}
+
+}  // namespace aafkv

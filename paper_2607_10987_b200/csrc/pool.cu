@@ -1,0 +1,696 @@
+// Host side of libaafkv.so: the C ABI declared in include/aaf_kv.h.
+//
+// The host object mirrors only what it can know without asking the device: which handles are
+// live and how many tokens each holds (every length is a function of the call sequence), plus a
+// guaranteed lower bound of the free-block count.  Block ids, reference counts and the ring live
+// on the device.  A call validates everything against the mirror, writes its argument records
+// into a pinned ring the planners read directly, and launches: planner kernel(s) then the copy
+// engine.  The device's free count is read back (one synchronising 16-byte copy) only when the
+// lower bound cannot prove that a call fits, so out-of-blocks is reported exactly and
+// synchronously without a sync on the common path.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "aafkv_internal.h"
+
+using namespace aafkv;
+
+namespace {
+
+constexpr int ARG_SLOTS = 16;
+
+struct Layout {
+    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, total;
+    int max_pieces, max_batch;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool geometry_ok(const aaf_kv_pool_desc *d) {
+    if (!d || d->struct_size != sizeof(aaf_kv_pool_desc) || d->abi_version != AAF_KV_ABI_VERSION) return false;
+    if (d->n_layers < 1 || d->n_kv_heads < 1 || d->head_dim < 1 || d->block_size < 1 || d->elt_bytes < 1) return false;
+    if (d->n_blocks < 1 || d->max_ctx < 1 || d->max_blocks_per_ctx < 1 || d->max_batch < 0) return false;
+    const long long row = (long long)d->n_kv_heads * d->head_dim * d->elt_bytes;
+    if (row % 16 != 0) return false;
+    if (row * d->block_size > (1ll << 30)) return false;  // a run must fit the 32-bit piece size
+    if ((long long)d->max_ctx * d->max_blocks_per_ctx > (1ll << 31)) return false;
+    return true;
+}
+
+Layout make_layout(const aaf_kv_pool_desc *d) {
+    Layout L{};
+    L.max_batch = d->max_batch > 0 ? d->max_batch : 1024;
+    L.max_pieces = 2 * d->max_blocks_per_ctx + 4 * L.max_batch + 64;
+    size_t off = 0;
+    L.ctl = off; off = align_up(off + sizeof(DevCtl), 256);
+    L.refcount = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
+    L.ring = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
+    L.last_pos = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
+    L.tables = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx * d->max_blocks_per_ctx, 256);
+    L.pieces = off; off = align_up(off + sizeof(Piece) * (size_t)L.max_pieces, 256);
+    L.scratch = off; off = align_up(off + sizeof(int) * 3 * (size_t)L.max_batch, 256);
+    L.total = off;
+    return L;
+}
+
+struct TimedLaunch {
+    cudaEvent_t start, stop;
+    int cls;
+};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct aaf_kv_pool {
+    aaf_kv_pool_desc desc;
+    Geom g;
+    DevState s;
+    Layout lay;
+    int device = 0, sm_count = 148;
+    std::vector<long long> len;  // tokens per handle, -1 = free
+    int live_ctx = 0;
+    long long free_lb = 0;       // guaranteed lower bound of the device's free-block count
+    cudaStream_t last_stream = nullptr;
+    // pinned argument ring
+    char *args = nullptr;
+    size_t slot_bytes = 0;
+    int next_slot = 0;
+    cudaEvent_t slot_ev[ARG_SLOTS] = {};
+    bool slot_busy[ARG_SLOTS] = {};
+    int cur_slot = -1;
+    // knobs and counters
+    int engine = AAF_ENGINE_AUTO;
+    bool timing = false;
+    long long copy_launches[AAF_OP_CLASSES] = {};
+    long long meta_launches = 0;
+    double copy_ms[AAF_OP_CLASSES] = {};
+    long long timed_launches[AAF_OP_CLASSES] = {};
+    std::vector<TimedLaunch> pending;
+    std::vector<cudaEvent_t> spare_events;
+};
+
+namespace {
+
+long long nblk_of(const aaf_kv_pool *p, long long tokens) { return (tokens + p->g.BS - 1) / p->g.BS; }
+bool is_live(const aaf_kv_pool *p, int c) { return c >= 0 && c < p->g.max_ctx && p->len[c] >= 0; }
+bool aligned16(const void *q) { return q && (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
+long long bpt_of(const aaf_kv_pool *p) { return 2ll * p->g.L * p->g.row; }
+
+// next pinned argument slot; waits (host side) until the device has finished reading its last use
+char *acquire_args(aaf_kv_pool *p) {
+    const int sl = p->next_slot;
+    p->next_slot = (sl + 1) % ARG_SLOTS;
+    if (p->slot_busy[sl]) {
+        cudaEventSynchronize(p->slot_ev[sl]);
+        p->slot_busy[sl] = false;
+    }
+    p->cur_slot = sl;
+    return p->args + (size_t)sl * p->slot_bytes;
+}
+void release_args(aaf_kv_pool *p, cudaStream_t st) {
+    if (p->cur_slot < 0) return;
+    cudaEventRecord(p->slot_ev[p->cur_slot], st);
+    p->slot_busy[p->cur_slot] = true;
+    p->cur_slot = -1;
+}
+
+// exact free-block count: synchronises the stream and reads the ring counters
+int refresh_free(aaf_kv_pool *p, cudaStream_t st) {
+    unsigned long long ht[2];
+    if (cudaStreamSynchronize(st) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaMemcpy(ht, p->s.ctl, sizeof(ht), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
+    p->free_lb = (long long)(ht[1] - ht[0]);
+    return AAF_OK;
+}
+int ensure_free(aaf_kv_pool *p, long long need, cudaStream_t st) {
+    if (p->free_lb >= need) return AAF_OK;
+    const int rc = refresh_free(p, st);
+    if (rc != AAF_OK) return rc;
+    return p->free_lb >= need ? AAF_OK : AAF_ERR_OOM_BLOCKS;
+}
+
+int smallest_free_ctx(const aaf_kv_pool *p, int start = 0) {
+    for (int c = start; c < p->g.max_ctx; ++c)
+        if (p->len[c] < 0) return c;
+    return -1;
+}
+
+cudaEvent_t get_event(aaf_kv_pool *p) {
+    if (!p->spare_events.empty()) {
+        cudaEvent_t e = p->spare_events.back();
+        p->spare_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+void drain_timing(aaf_kv_pool *p) {
+    for (auto &t : p->pending) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(t.stop) == cudaSuccess && cudaEventElapsedTime(&ms, t.start, t.stop) == cudaSuccess) {
+            p->copy_ms[t.cls] += ms;
+            p->timed_launches[t.cls] += 1;
+        }
+        p->spare_events.push_back(t.start);
+        p->spare_events.push_back(t.stop);
+    }
+    p->pending.clear();
+}
+
+// copy-engine launch for one operator class over planes [plane0, plane0 + n_planes)
+int run_copy(aaf_kv_pool *p, int cls, int n_slots, int plane0, int n_planes, cudaStream_t st) {
+    if (n_slots <= 0) return AAF_OK;
+    TimedLaunch t{};
+    if (p->timing) {
+        t.start = get_event(p);
+        t.stop = get_event(p);
+        t.cls = cls;
+        cudaEventRecord(t.start, st);
+    }
+    const cudaError_t e = launch_copy(p->engine, p->g, p->s, n_slots, plane0, n_planes, p->sm_count, st);
+    if (p->timing) {
+        cudaEventRecord(t.stop, st);
+        p->pending.push_back(t);
+        if (p->pending.size() > 4096) drain_timing(p);
+    }
+    p->copy_launches[cls] += 1;
+    return e == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
+}
+
+void fill_desc(const aaf_kv_pool *p, aaf_kv_xfer_desc *d, long long pos_start, long long n) {
+    d->model_id = p->desc.model_id;
+    d->config_hash = p->desc.config_hash;
+    d->n_layers = p->g.L; d->n_kv_heads = p->g.H; d->head_dim = p->g.D; d->elt_bytes = p->g.E;
+    d->pos_start = pos_start;
+    d->n_tokens = n;
+}
+
+// Compat(S_a, S_b) = 1[M_a = M_b] * 1[Theta_a = Theta_b] (Sec. 3.2); positions are carried, not enforced
+bool compatible(const aaf_kv_pool *p, const aaf_kv_xfer_desc *d) {
+    return d->model_id == p->desc.model_id && d->config_hash == p->desc.config_hash && d->n_layers == p->g.L &&
+           d->n_kv_heads == p->g.H && d->head_dim == p->g.D && d->elt_bytes == p->g.E;
+}
+
+int materialize_impl(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void *dst_dev, size_t dst_bytes,
+                     aaf_kv_xfer_desc *out_desc, cudaStream_t st) {
+    if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
+    if (!aligned16(dst_dev) || t0 < 0 || t0 >= t1 || t1 > p->len[ctx]) return AAF_ERR_INVALID_ARG;
+    const long long n = t1 - t0;
+    if ((unsigned long long)dst_bytes < (unsigned long long)(n * bpt_of(p))) return AAF_ERR_DST_TOO_SMALL;
+    p->last_stream = st;
+    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(dst_dev), st) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    const int n_slots = (int)((t1 - 1) / p->g.BS - t0 / p->g.BS + 1);
+    const int rc = run_copy(p, AAF_OP_MATERIALIZE, n_slots, 0, 2 * p->g.L, st);
+    if (rc == AAF_OK && out_desc) fill_desc(p, out_desc, t0, n);
+    return rc;
+}
+
+int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
+                cudaStream_t st, const void *src_host) {
+    if (!desc || !out_ctx || !aligned16(src_dev)) return AAF_ERR_INVALID_ARG;
+    if (!compatible(p, desc)) return AAF_ERR_INCOMPAT;
+    const long long n = desc->n_tokens;
+    if (n < 1) return AAF_ERR_INVALID_ARG;
+    const long long nb = nblk_of(p, n);
+    if (nb > p->g.max_blk) return AAF_ERR_TOO_LONG;
+    const int c = smallest_free_ctx(p);
+    if (c < 0) return AAF_ERR_OOM_CTX;
+    const int rc0 = ensure_free(p, nb, st);
+    if (rc0 != AAF_OK) return rc0;
+    p->last_stream = st;
+    if (src_host) {
+        if (cudaMemcpyAsync(const_cast<void *>(src_dev), src_host, (size_t)(n * bpt_of(p)), cudaMemcpyHostToDevice,
+                            st) != cudaSuccess)
+            return AAF_ERR_CUDA;
+    }
+    if (launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(src_dev), st) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    p->free_lb -= nb;
+    p->len[c] = n;
+    p->live_ctx += 1;
+    *out_ctx = c;
+    return run_copy(p, AAF_OP_IMPORT, (int)nb, 0, 2 * p->g.L, st);
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+size_t aaf_kv_pool_workspace_bytes(const aaf_kv_pool_desc *desc) {
+    if (!geometry_ok(desc)) return 0;
+    return make_layout(desc).total;
+}
+
+int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
+    if (!out) return AAF_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!geometry_ok(desc)) return AAF_ERR_INVALID_ARG;
+    const Layout lay = make_layout(desc);
+    const long long row = (long long)desc->n_kv_heads * desc->head_dim * desc->elt_bytes;
+    const long long run = row * desc->block_size;
+    if (!aligned16(desc->pool_base) || !desc->workspace || (reinterpret_cast<uintptr_t>(desc->workspace) & 255u))
+        return AAF_ERR_INVALID_ARG;
+    if (desc->layer_stride_bytes % 16 != 0 || desc->layer_stride_bytes < (size_t)(2 * run * desc->n_blocks))
+        return AAF_ERR_INVALID_ARG;
+    if (desc->workspace_bytes < lay.total) return AAF_ERR_INVALID_ARG;
+    std::vector<int> ring((size_t)desc->n_blocks);
+    if (desc->free_order) {
+        std::vector<char> seen((size_t)desc->n_blocks, 0);
+        for (int i = 0; i < desc->n_blocks; ++i) {
+            const int b = desc->free_order[i];
+            if (b < 0 || b >= desc->n_blocks || seen[(size_t)b]) return AAF_ERR_INVALID_ARG;
+            seen[(size_t)b] = 1;
+            ring[(size_t)i] = b;
+        }
+    } else {
+        for (int i = 0; i < desc->n_blocks; ++i) ring[(size_t)i] = i;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || desc->device < 0 || desc->device >= ndev) return AAF_ERR_CUDA;
+
+    aaf_kv_pool *p = new (std::nothrow) aaf_kv_pool();
+    if (!p) return AAF_ERR_INVALID_ARG;
+    p->desc = *desc;
+    p->desc.free_order = nullptr;
+    p->lay = lay;
+    p->device = desc->device;
+    DeviceGuard guard(p->device);
+    p->g.L = desc->n_layers; p->g.H = desc->n_kv_heads; p->g.D = desc->head_dim; p->g.BS = desc->block_size;
+    p->g.E = desc->elt_bytes; p->g.NB = desc->n_blocks; p->g.max_ctx = desc->max_ctx;
+    p->g.max_blk = desc->max_blocks_per_ctx;
+    p->g.row = row; p->g.run = run; p->g.layer_stride = (long long)desc->layer_stride_bytes;
+    p->g.pool = static_cast<char *>(desc->pool_base);
+    char *ws = static_cast<char *>(desc->workspace);
+    p->s.ctl = reinterpret_cast<DevCtl *>(ws + lay.ctl);
+    p->s.refcount = reinterpret_cast<int *>(ws + lay.refcount);
+    p->s.ring = reinterpret_cast<int *>(ws + lay.ring);
+    p->s.last_pos = reinterpret_cast<int *>(ws + lay.last_pos);
+    p->s.tables = reinterpret_cast<int *>(ws + lay.tables);
+    p->s.pieces = reinterpret_cast<Piece *>(ws + lay.pieces);
+    p->s.scratch = reinterpret_cast<int *>(ws + lay.scratch);
+    p->len.assign((size_t)desc->max_ctx, -1);
+    p->free_lb = desc->n_blocks;
+
+    bool ok = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) == cudaSuccess;
+    ok = ok && copy_engine_init(p->device) == cudaSuccess;
+    p->slot_bytes = align_up(48 * (size_t)lay.max_batch + 256, 256);
+    ok = ok && cudaHostAlloc(reinterpret_cast<void **>(&p->args), p->slot_bytes * ARG_SLOTS, cudaHostAllocMapped) ==
+                   cudaSuccess;
+    for (int i = 0; ok && i < ARG_SLOTS; ++i)
+        ok = cudaEventCreateWithFlags(&p->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    // device state: counters, reference counts 0, ring, evict scratch -1
+    DevCtl ctl;
+    memset(&ctl, 0, sizeof(ctl));
+    ctl.tail = (unsigned long long)desc->n_blocks;
+    ok = ok && cudaMemset(ws, 0, lay.tables) == cudaSuccess;
+    ok = ok && cudaMemcpy(p->s.ctl, &ctl, sizeof(ctl), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(p->s.ring, ring.data(), sizeof(int) * ring.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(p->s.last_pos, 0xff, sizeof(int) * (size_t)desc->n_blocks) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        aaf_kv_pool_destroy(p);
+        return AAF_ERR_CUDA;
+    }
+    *out = p;
+    return AAF_OK;
+}
+
+int aaf_kv_pool_destroy(aaf_kv_pool *p) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (p->last_stream || !p->pending.empty()) cudaStreamSynchronize(p->last_stream);
+    for (auto &t : p->pending) {
+        cudaEventDestroy(t.start);
+        cudaEventDestroy(t.stop);
+    }
+    for (auto e : p->spare_events) cudaEventDestroy(e);
+    for (int i = 0; i < ARG_SLOTS; ++i)
+        if (p->slot_ev[i]) cudaEventDestroy(p->slot_ev[i]);
+    if (p->args) cudaFreeHost(p->args);
+    delete p;
+    return AAF_OK;
+}
+
+int aaf_kv_materialize(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_dev,
+                       size_t dst_bytes, aaf_kv_xfer_desc *out_desc, void *stream) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    return materialize_impl(p, ctx, tok_begin, tok_end, dst_dev, dst_bytes, out_desc,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int aaf_kv_materialize_host(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_host,
+                            size_t dst_bytes, void *staging_dev, size_t staging_bytes, aaf_kv_xfer_desc *out_desc,
+                            void *stream) {
+    if (!p || !dst_host) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (is_live(p, ctx) && tok_begin >= 0 && tok_begin < tok_end &&
+        (unsigned long long)dst_bytes < (unsigned long long)((tok_end - tok_begin) * bpt_of(p)))
+        return AAF_ERR_DST_TOO_SMALL;
+    const int rc = materialize_impl(p, ctx, tok_begin, tok_end, staging_dev, staging_bytes, out_desc, st);
+    if (rc != AAF_OK) return rc;
+    const size_t bytes = (size_t)((tok_end - tok_begin) * bpt_of(p));
+    return cudaMemcpyAsync(dst_host, staging_dev, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess ? AAF_OK
+                                                                                                   : AAF_ERR_CUDA;
+}
+
+int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
+                  void *stream) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    return import_impl(p, src_dev, desc, out_ctx, static_cast<cudaStream_t>(stream), nullptr);
+}
+
+int aaf_kv_import_host(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
+                       size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream) {
+    if (!p || !src_host || !desc) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (desc->n_tokens >= 1 && (unsigned long long)staging_bytes < (unsigned long long)(desc->n_tokens * bpt_of(p)))
+        return AAF_ERR_DST_TOO_SMALL;
+    return import_impl(p, staging_dev, desc, out_ctx, static_cast<cudaStream_t>(stream), src_host);
+}
+
+int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream) {
+    if (!p || !out_children || k < 1) return AAF_ERR_INVALID_ARG;
+    if (!is_live(p, parent)) return AAF_ERR_BAD_CTX;
+    if (k > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    if (p->g.max_ctx - p->live_ctx < k) return AAF_ERR_OOM_CTX;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    int *children = reinterpret_cast<int *>(acquire_args(p));
+    int c = -1;
+    for (int j = 0; j < k; ++j) {
+        c = smallest_free_ctx(p, c + 1);
+        children[j] = c;
+    }
+    const long long T = p->len[parent];
+    const cudaError_t e = launch_fork(p->g, p->s, parent, (int)nblk_of(p, T), k, children, st);
+    release_args(p, st);
+    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    for (int j = 0; j < k; ++j) {
+        p->len[children[j]] = T;
+        out_children[j] = children[j];
+    }
+    p->live_ctx += k;
+    return AAF_OK;
+}
+
+int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
+                  const void *const *src_dev, void *stream) {
+    if (!p || n < 1 || !ctxs || !n_new || !src_dev) return AAF_ERR_INVALID_ARG;
+    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    for (int i = 0; i < n; ++i) {
+        if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
+        if (n_new[i] < 1 || !aligned16(src_dev[i])) return AAF_ERR_INVALID_ARG;
+    }
+    {
+        std::vector<int> sorted(ctxs, ctxs + n);
+        std::sort(sorted.begin(), sorted.end());
+        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AAF_ERR_INVALID_ARG;
+    }
+    const int BS = p->g.BS;
+    long long worst = 0, slots = 0;
+    for (int i = 0; i < n; ++i) {
+        const long long T = p->len[ctxs[i]];
+        if (nblk_of(p, T + n_new[i]) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+        worst += (T % BS ? 1 : 0) + nblk_of(p, T + n_new[i]) - nblk_of(p, T);
+        slots += 1 + nblk_of(p, T + n_new[i]) - T / BS;
+    }
+    if (slots > p->lay.max_pieces) return AAF_ERR_TOO_MANY;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+
+    AppendEntry *ent = reinterpret_cast<AppendEntry *>(acquire_args(p));
+    int off = 0;
+    for (int i = 0; i < n; ++i) {
+        const long long T = p->len[ctxs[i]];
+        ent[i].src = static_cast<const char *>(src_dev[i]);
+        ent[i].T = T;
+        ent[i].ctx = ctxs[i];
+        ent[i].n_new = n_new[i];
+        ent[i].piece_off = off;
+        ent[i].pad = 0;
+        off += (int)(1 + nblk_of(p, T + n_new[i]) - T / BS);
+    }
+    long long charge = worst;  // what the lower bound is reduced by
+    if (p->free_lb < worst) {
+        int rc = refresh_free(p, st);
+        if (rc == AAF_OK && p->free_lb < worst) {
+            // the worst case does not fit: ask the planner (dry run) how many blocks the batch really
+            // needs; only tail blocks that are still shared are copied
+            unsigned long long need = 0;
+            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, st) != cudaSuccess ||
+                cudaStreamSynchronize(st) != cudaSuccess ||
+                cudaMemcpy(&need, &p->s.ctl->probe_need, sizeof(need), cudaMemcpyDeviceToHost) != cudaSuccess)
+                rc = AAF_ERR_CUDA;
+            else if ((long long)need > p->free_lb)
+                rc = AAF_ERR_OOM_BLOCKS;
+            p->meta_launches += 1;
+            charge = (long long)need;
+        }
+        if (rc != AAF_OK) {
+            release_args(p, st);
+            return rc;
+        }
+    }
+    const cudaError_t e = launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 0, st);
+    release_args(p, st);
+    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    p->free_lb -= charge;
+    for (int i = 0; i < n; ++i) p->len[ctxs[i]] += n_new[i];
+    return run_copy(p, AAF_OP_APPEND, (int)slots, 0, 2 * p->g.L, st);
+}
+
+int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
+                   void *stream) {
+    if (!p || m < 1 || !segs || !out_ctx || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
+    if (m > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    for (int i = 0; i < m; ++i)
+        if (!is_live(p, segs[i])) return AAF_ERR_BAD_CTX;
+    const bool copy_all = (flags & AAF_COMPOSE_COPY_ALL) != 0;
+    const int BS = p->g.BS;
+    // everything but the block ids follows from the lengths
+    std::vector<ComposeSeg> rec((size_t)m);
+    long long off = 0, fresh = 0, work = 0, slots = 0, tbl = 0;
+    for (int i = 0; i < m; ++i) {
+        const long long T = p->len[segs[i]];
+        ComposeSeg &r = rec[(size_t)i];
+        memset(&r, 0, sizeof(r));
+        r.T = T; r.off = off; r.ctx = segs[i];
+        r.work_off = (int)work; r.fresh_start = (int)fresh; r.piece_off = (int)slots;
+        if (!copy_all && off % BS == 0) {
+            r.mode = 0;
+            r.share_tail = (i == m - 1);
+            r.dst_tbl_start = (int)tbl;
+            const long long items = nblk_of(p, T);
+            work += items;
+            if (T % BS && i != m - 1) { fresh += 1; slots += 1; }
+        } else {
+            r.mode = 1;
+            const long long items = (off + T - 1) / BS - off / BS + 1;
+            work += items;
+            slots += 2 * items;
+            fresh += nblk_of(p, off + T) - nblk_of(p, off);
+        }
+        off += T;
+        tbl = nblk_of(p, off);
+    }
+    if (nblk_of(p, off) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+    if (slots > p->lay.max_pieces) return AAF_ERR_TOO_MANY;
+    const int c = smallest_free_ctx(p);
+    if (c < 0) return AAF_ERR_OOM_CTX;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int rc0 = ensure_free(p, fresh, st);
+    if (rc0 != AAF_OK) return rc0;
+    p->last_stream = st;
+    ComposeSeg *dev_rec = reinterpret_cast<ComposeSeg *>(acquire_args(p));
+    memcpy(dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
+    const cudaError_t e =
+        launch_plan_compose(p->g, p->s, dev_rec, m, (int)work, (int)fresh, (int)slots, c, st);
+    release_args(p, st);
+    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    p->free_lb -= fresh;
+    p->len[c] = off;
+    p->live_ctx += 1;
+    *out_ctx = c;
+    return run_copy(p, AAF_OP_COMPOSE, (int)slots, 0, 2 * p->g.L, st);
+}
+
+int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {
+    if (!p || n < 1 || !ctxs) return AAF_ERR_INVALID_ARG;
+    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    for (int i = 0; i < n; ++i)
+        if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
+    {
+        std::vector<int> sorted(ctxs, ctxs + n);
+        std::sort(sorted.begin(), sorted.end());
+        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AAF_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    EvictArgs *a = reinterpret_cast<EvictArgs *>(acquire_args(p));
+    int *ctx = reinterpret_cast<int *>(a + 1);
+    int *ent_off = ctx + n;
+    long long total = 0;
+    for (int i = 0; i < n; ++i) {
+        ctx[i] = ctxs[i];
+        ent_off[i] = (int)total;
+        total += nblk_of(p, p->len[ctxs[i]]);
+    }
+    ent_off[n] = (int)total;
+    a->n = n;
+    a->total = (int)total;
+    const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, st);
+    release_args(p, st);
+    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->meta_launches += 2;
+    for (int i = 0; i < n; ++i) p->len[ctxs[i]] = -1;
+    p->live_ctx -= n;
+    return AAF_OK;  // the lower bound of the free count stays valid: evict only adds free blocks
+}
+
+int aaf_kv_ctx_len(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t *n_tokens) {
+    if (!p || !n_tokens) return AAF_ERR_INVALID_ARG;
+    if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
+    *n_tokens = p->len[ctx];
+    return AAF_OK;
+}
+
+int aaf_kv_get_table(aaf_kv_pool *p, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks) {
+    if (!p || !host_out || !n_blocks) return AAF_ERR_INVALID_ARG;
+    if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
+    const long long nb = nblk_of(p, p->len[ctx]);
+    if (cap < nb) return AAF_ERR_DST_TOO_SMALL;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaMemcpy(host_out, p->s.tables + (long long)ctx * p->g.max_blk, sizeof(int) * (size_t)nb,
+                   cudaMemcpyDeviceToHost) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    *n_blocks = (int32_t)nb;
+    return AAF_OK;
+}
+
+int aaf_kv_get_refcounts(aaf_kv_pool *p, int32_t *host_out) {
+    if (!p || !host_out) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    return cudaMemcpy(host_out, p->s.refcount, sizeof(int) * (size_t)p->g.NB, cudaMemcpyDeviceToHost) == cudaSuccess
+               ? AAF_OK
+               : AAF_ERR_CUDA;
+}
+
+int aaf_kv_get_free_list(aaf_kv_pool *p, int32_t *host_out, int32_t *n_free) {
+    if (!p || !host_out || !n_free) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    unsigned long long ht[2];
+    std::vector<int> ring((size_t)p->g.NB);
+    if (cudaMemcpy(ht, p->s.ctl, sizeof(ht), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(ring.data(), p->s.ring, sizeof(int) * ring.size(), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    const unsigned long long f = ht[1] - ht[0];
+    if (f > (unsigned long long)p->g.NB) return AAF_ERR_CORRUPT;
+    for (unsigned long long i = 0; i < f; ++i) host_out[i] = ring[(size_t)((ht[0] + i) % (unsigned long long)p->g.NB)];
+    *n_free = (int32_t)f;
+    p->free_lb = (long long)f;
+    return AAF_OK;
+}
+
+int aaf_kv_pool_stats(aaf_kv_pool *p, aaf_kv_stats *out) {
+    if (!p || !out) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    drain_timing(p);
+    DevCtl ctl;
+    if (cudaMemcpy(&ctl, p->s.ctl, sizeof(ctl), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
+    memset(out, 0, sizeof(*out));
+    out->free_blocks = (int64_t)(ctl.tail - ctl.head);
+    out->live_blocks = p->g.NB - out->free_blocks;
+    out->peak_live_blocks = ctl.peak_live;
+    out->live_ctx = p->live_ctx;
+    out->cow_count = (int64_t)ctl.cow_count;
+    out->payload_bytes = (int64_t)ctl.payload_bytes;
+    out->meta_launches = p->meta_launches;
+    for (int i = 0; i < AAF_OP_CLASSES; ++i) {
+        out->copy_launches[i] = p->copy_launches[i];
+        out->copy_ms[i] = p->copy_ms[i];
+        out->timed_launches[i] = p->timed_launches[i];
+    }
+    p->free_lb = out->free_blocks;
+    return AAF_OK;
+}
+
+int aaf_kv_sync_status(aaf_kv_pool *p) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    int st[2] = {0, 0};
+    if (cudaMemcpy(st, &p->s.ctl->status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
+    if (st[0] != 0) {
+        const int zero[2] = {0, 0};
+        cudaMemcpy(&p->s.ctl->status, zero, sizeof(zero), cudaMemcpyHostToDevice);
+    }
+    return st[0];
+}
+
+int aaf_kv_set_copy_engine(aaf_kv_pool *p, int engine) {
+    if (!p || engine < AAF_ENGINE_AUTO || engine > AAF_ENGINE_BULK) return AAF_ERR_INVALID_ARG;
+    p->engine = engine;
+    return AAF_OK;
+}
+
+int aaf_kv_set_timing(aaf_kv_pool *p, int enable) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    p->timing = enable != 0;
+    return AAF_OK;
+}
+
+const char *aaf_kv_strerror(int status) {
+    switch (status) {
+        case AAF_OK: return "ok";
+        case AAF_ERR_INVALID_ARG: return "invalid argument";
+        case AAF_ERR_BAD_CTX: return "not a live context";
+        case AAF_ERR_OOM_BLOCKS: return "out of free blocks";
+        case AAF_ERR_OOM_CTX: return "out of context handles";
+        case AAF_ERR_TOO_LONG: return "context would exceed max_blocks_per_ctx";
+        case AAF_ERR_INCOMPAT: return "descriptor incompatible with the pool";
+        case AAF_ERR_DST_TOO_SMALL: return "destination too small";
+        case AAF_ERR_CUDA: return "CUDA runtime error";
+        case AAF_ERR_CORRUPT: return "device found pool metadata inconsistent";
+        case AAF_ERR_TIMEOUT: return "bounded device wait expired";
+        case AAF_ERR_TOO_MANY: return "batch exceeds max_batch or the piece capacity";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -160,3 +160,57 @@ def expected_bytes(seed: int, g: Geometry, tokens, layers=None) -> np.ndarray:
                 idx = (((l * 2 + kv) * nn[sel] + tt[sel]) * hd)[:, None] + lane[None, :]
                 out[i, kv, sel] = fill.fill_np_at(seed, int(s), idx)
     return out.view(np.uint8).reshape(len(layers), 2, len(tokens), g.row)
+
+
+class GpuBackend:
+    """The CUDA library (through its Python binding) behind the replay-backend interface."""
+
+    def __init__(self, g: Geometry, seed: int, free_order=None, engine: int = 0, init_fill=True, max_batch=0):
+        import torch
+
+        from paper_2607_10987_b200 import KVPool
+
+        self.g, self.torch = g, torch
+        self.o = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, g.n_blocks, g.max_ctx,
+                        g.max_blocks_per_ctx, free_order=free_order, max_batch=max_batch)
+        self.o.set_copy_engine(engine)
+        if init_fill:
+            fill.fill_torch(seed, 0, 0, g.pool_bytes // 2, self.o.device, out=self.o.pool.view(torch.int16))
+        torch.cuda.synchronize()
+
+    def payload(self, seed, stream, n):
+        g = self.g
+        return fill.fill_torch(seed, stream, 0, g.n_layers * 2 * n * g.row // 2, self.o.device).view(self.torch.uint8)
+
+    def imp(self, buf, n):
+        return self.o.imp(buf, n)
+
+    def materialize(self, c, t0, t1):
+        return self.o.materialize(c, t0, t1)
+
+    def fork(self, c, k):
+        return self.o.fork(c, k)
+
+    def append(self, ctxs, n_new, bufs):
+        return self.o.append(ctxs, n_new, bufs)
+
+    def compose(self, ctxs, flags):
+        return self.o.compose(ctxs, flags)
+
+    def evict(self, ctxs):
+        return self.o.evict(ctxs)
+
+    def snapshot(self):
+        return snapshot(self.o)
+
+    def pool_layers(self, layers) -> np.ndarray:
+        """uint8 [len(layers), NB, 2, BS, row] copy of the given layers of the device pool."""
+        g = self.g
+        v = self.o.pool[: g.pool_bytes].view(g.n_layers, g.n_blocks, 2, g.block_size, g.row)
+        return v[list(layers)].cpu().numpy()
+
+    def buf_layers(self, buf, n, layers) -> np.ndarray:
+        """uint8 [len(layers), 2, n, row] copy of the given layers of a device transfer buffer."""
+        g = self.g
+        v = buf[: n * g.bpt].view(g.n_layers, 2, n, g.row)
+        return v[list(layers)].cpu().numpy()

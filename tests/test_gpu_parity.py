@@ -1,0 +1,166 @@
+"""Parity of the CUDA library against the CPU oracle, element by element, through the C ABI.
+
+Bit-exact bar: every materialised byte, every pool byte of the compared layers (stale slots
+included), all block tables, token counts, reference counts and the free list in ring order.
+"""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from tests.helpers import GpuBackend, OracleBackend, check_conservation
+from workloads import configs
+from workloads.configs import Geometry
+from workloads.replay import replay
+
+pytestmark = pytest.mark.gpu
+
+VEC, BULK = 1, 2
+
+
+def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
+    """Replays ops on the GPU library and on the oracle side by side and compares after every op."""
+    layers = list(range(g.n_layers)) if layers is None else list(layers)
+    order = configs.free_order(seed, g.n_blocks) if order is None else order
+    gpu = GpuBackend(g, seed, free_order=order, engine=engine, max_batch=max_batch)
+    cpu = OracleBackend(g, seed, layers=layers, free_order=order)
+    for (i, op, st_g, res_g, _), (_, _, st_c, res_c, _) in zip(replay(ops, gpu, seed), replay(ops, cpu, seed)):
+        assert st_g == st_c, (i, op, st_g, st_c)
+        assert gpu.snapshot() == cpu.snapshot(), (i, op)
+        if op["op"] == "materialize" and st_c == 0:
+            n = op["t1"] - op["t0"]
+            assert np.array_equal(gpu.buf_layers(res_g, n, layers).reshape(-1), res_c), (i, op)
+    assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view()), "pool image differs"
+    assert gpu.o.sync_status() == 0
+    gs, cs = gpu.o.stats(), cpu.o.stats()
+    for k in ("free_blocks", "live_blocks", "peak_live_blocks", "live_ctx", "cow_count"):
+        assert gs[k] == cs[k], (k, gs[k], cs[k])
+    assert gs["payload_bytes"] == cs["rows_copied"] * g.row * g.n_layers // len(layers)
+    return gpu, cpu
+
+
+@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("unaligned", [False, True])
+def test_config1_tiny_pool(engine, unaligned):
+    g, seed, ops = configs.config1(unaligned)
+    gpu, cpu = lockstep(g, seed, ops, engine=engine)
+    assert gpu.o.stats()["cow_count"] == (4 if unaligned else 0)
+    assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
+
+
+# odd geometry: row = 3*40*2 = 240 bytes (not a power of two), run = 1680 bytes, several chunks per
+# launch and a ragged tail everywhere
+ODD = Geometry(3, 3, 40, 7, 2, 48, 10, 24)
+
+
+def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
+    """Random operators chosen against the oracle's current state, applied to both sides and compared
+    after every operator.  Lengths and counts are drawn so that out-of-blocks, out-of-handles and
+    too-long failures occur naturally; a few operators are made invalid on purpose (dead handle,
+    duplicate context, empty range).  Failures must be identical and change nothing."""
+    rng = np.random.default_rng(seed)
+    order = configs.free_order(seed, g.n_blocks)
+    gpu = GpuBackend(g, seed, free_order=order, engine=engine)
+    cpu = OracleBackend(g, seed, free_order=order)
+    layers = list(range(g.n_layers))
+    stream = 1
+    outcomes = []
+    for i in range(n_ops):
+        live = cpu.o.live_ctxs()
+        kind = str(rng.choice(["import", "fork", "append", "compose", "evict", "materialize", "roundtrip"],
+                              p=[0.16, 0.12, 0.26, 0.14, 0.12, 0.14, 0.06]))
+        if not live:
+            kind = "import"
+        pick = lambda: int(rng.choice(live)) if rng.random() > 0.04 else int(rng.integers(0, g.max_ctx))
+        both = (gpu, cpu)
+        if kind == "import":
+            n = int(rng.integers(1, 6 * g.block_size))
+            res = [be.imp(be.payload(seed, stream, n), n) for be in both]
+            stream += 1
+        elif kind == "fork":
+            c, k = pick(), int(rng.integers(0, 4))
+            res = [be.fork(c, k) for be in both]
+        elif kind == "append":
+            m = int(rng.integers(1, 4))
+            who = [pick() for _ in range(m)]  # duplicates possible -> INVALID_ARG
+            nn = [int(rng.integers(1, 3 * g.block_size)) for _ in who]
+            res = [be.append(who, nn, [be.payload(seed, stream + j, n) for j, n in enumerate(nn)]) for be in both]
+            stream += m
+        elif kind == "compose":
+            segs = [pick() for _ in range(int(rng.integers(1, 4)))]
+            fl = int(rng.integers(0, 2))
+            res = [be.compose(segs, fl) for be in both]
+        elif kind == "evict":
+            who = [pick() for _ in range(int(rng.integers(1, 3)))]
+            res = [be.evict(who) for be in both]
+        else:
+            c = pick()
+            T = cpu.o.ctx_len(c) or 4
+            a = int(rng.integers(0, T))
+            b = int(rng.integers(a, T + 1)) if kind == "materialize" else T  # a == b -> INVALID_ARG
+            a = a if kind == "materialize" else 0
+            res = [be.materialize(c, a, b) for be in both]
+            if res[1][0] == 0:
+                assert np.array_equal(gpu.buf_layers(res[0][1], b - a, layers).reshape(-1), res[1][1]), (i, kind)
+                if kind == "roundtrip":
+                    res = [gpu.imp(res[0][1], b - a), cpu.imp(res[1][1], b - a)]
+        (st_g, r_g), (st_c, r_c) = res
+        assert st_g == st_c, (i, kind, st_g, st_c)
+        if kind != "materialize":
+            assert r_g == r_c or kind == "roundtrip" and st_c == 0 and r_g == r_c, (i, kind, r_g, r_c)
+        snap = cpu.snapshot()
+        assert gpu.snapshot() == snap, (i, kind)
+        check_conservation(snap, g.n_blocks, g.block_size)
+        if i % 8 == 7:
+            assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view()), (i, kind)
+        outcomes.append((kind, st_c))
+    assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view())
+    assert gpu.o.sync_status() == 0
+    return outcomes
+
+
+@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_operator_sequences_on_odd_geometry(engine, seed):
+    outcomes = random_walk(ODD, 7000 + seed, 200, engine)
+    ok = {k for k, st in outcomes if st == 0}
+    assert ok >= {"import", "fork", "append", "compose", "evict", "materialize"}
+    failed = {st for _, st in outcomes if st < 0}
+    assert -3 in failed, "the walk should run out of blocks at least once"
+
+
+# 8B-shaped rows (2 KiB rows, 32 KiB runs) on a pool small enough for the oracle to hold all layers
+MID = Geometry(4, 8, 128, 16, 2, 1024, 24, 256)
+
+
+@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("unaligned", [False, True])
+def test_fanout_with_8b_rows(engine, unaligned):
+    T = 1019 if unaligned else 1024
+    ops = configs.fanout_ops(T, 6, 100, compose_pair=True, evict_all=True, roundtrip=True)
+    lockstep(MID, 4242, ops, engine=engine)
+
+
+def test_batched_append_equals_single_appends():
+    T = 1019
+    a = configs.fanout_ops(T, 6, 37, compose_pair=False, evict_all=False, roundtrip=False, batched_append=True)
+    b = configs.fanout_ops(T, 6, 37, compose_pair=False, evict_all=False, roundtrip=False, batched_append=False)
+    ga, _ = lockstep(MID, 99, a)
+    gb, _ = lockstep(MID, 99, b)
+    assert ga.snapshot() == gb.snapshot()
+    layers = list(range(MID.n_layers))
+    assert np.array_equal(ga.pool_layers(layers), gb.pool_layers(layers))
+
+
+@pytest.mark.parametrize("copy_all", [False, True])
+def test_compose_tree_small(copy_all):
+    g = Geometry(2, 8, 128, 16, 2, 2048, 40, 512)
+    g2, seed, ops, lens = configs.config3(g, copy_all=copy_all, lo=100, hi=400)
+    lockstep(g, seed, ops)
+
+
+def test_cow_stress_many_children():
+    g = Geometry(2, 8, 128, 16, 2, 1024, 300, 64)
+    ops = configs.cow_stress_ops(context_tokens=507, n_children=256)
+    gpu, cpu = lockstep(g, 5150, ops, max_batch=256)
+    assert gpu.o.stats()["cow_count"] == 256  # every child copies: the parent keeps the old tail
