@@ -56,6 +56,10 @@ def workload(name: str):
         g = configs.LLAMA70B
         return dict(name="llama3-70b-shaped KV, 32763-token context, 8 agents x 1024 tokens, unaligned (COW)", g=g,
                     seed=configs.SEED_BASE + 4, T=32763, agents=8, n_new=1024)
+    if name == "8b-small":  # same rows and runs as "8b" on a pool small enough for a full ncu capture
+        g = configs.Geometry(32, 8, 128, 16, 2, 2048, 16, 512)
+        return dict(name="llama3-8b-shaped KV rows, 2043-token context, 4 agents x 128 tokens, 2048-block pool", g=g,
+                    seed=configs.SEED_BASE + 2, T=2043, agents=4, n_new=128)
     if name == "tiny":
         g = configs.TINY
         return dict(name="tiny pool, 507-token context, 4 agents x 64 tokens", g=g, seed=configs.SEED_BASE + 1,
@@ -195,7 +199,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "tiny"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny"])
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST, 2 cp.async.bulk")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

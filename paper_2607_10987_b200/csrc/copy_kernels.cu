@@ -202,7 +202,7 @@ static int g_bulk_chunk = 16384;
 static int g_bulk_stages = 4;
 static int g_bulk_ctas_per_sm = 3;
 static int g_vec_unroll = 4;
-static int g_vec_ctas_per_sm = 8;
+static int g_vec_ctas_per_sm = 8;  // upper limit; the launch uses min(this, resident CTAs per SM)
 static int g_auto_engine = AAF_ENGINE_VEC;
 
 static int env_int(const char *name, int dflt, int lo, int hi) {
@@ -228,13 +228,27 @@ cudaError_t copy_engine_init(int device) {
                                 g_bulk_chunk * g_bulk_stages);
 }
 
+// resident CTAs per SM of a kernel, capped by the knob: the persistent grid must fit in ONE wave,
+// otherwise the CTAs of the second wave start when the first ones are done and the tail doubles
+template <typename K>
+static int resident_ctas(K kernel, int threads, size_t dyn_smem, int knob) {
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, threads, dyn_smem) != cudaSuccess || occ < 1) {
+        cudaGetLastError();
+        occ = 1;
+    }
+    return occ < knob ? occ : knob;
+}
+
 template <int UNROLL>
 static void launch_vec(const DevState &s, int n_slots, int plane0, int n_planes, long long run, int sm_count,
                        cudaStream_t st) {
     constexpr long long CHUNK = (long long)VEC_THREADS * UNROLL * 16;
+    static int ctas = 0;  // per template instance; the knobs are fixed after the first pool creation
+    if (ctas == 0) ctas = resident_ctas(copy_vec_kernel<UNROLL>, VEC_THREADS, 0, g_vec_ctas_per_sm);
     const int cpp = (int)((run + CHUNK - 1) / CHUNK);
     const long long total = (long long)n_slots * n_planes * cpp;
-    const long long cap = (long long)sm_count * g_vec_ctas_per_sm;
+    const long long cap = (long long)sm_count * ctas;
     const int grid = (int)(total < cap ? total : cap);
     copy_vec_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp);
 }
@@ -244,9 +258,12 @@ cudaError_t launch_copy(int engine, const Geom &g, const DevState &s, int n_slot
     if (n_slots <= 0 || n_planes <= 0) return cudaSuccess;
     if (engine == AAF_ENGINE_AUTO) engine = g_auto_engine;
     if (engine == AAF_ENGINE_BULK) {
+        static int ctas = 0;
+        if (ctas == 0)
+            ctas = resident_ctas(copy_bulk_kernel, 32, (size_t)g_bulk_chunk * g_bulk_stages, g_bulk_ctas_per_sm);
         const int cpp = (int)((g.run + g_bulk_chunk - 1) / g_bulk_chunk);
         const long long total = (long long)n_slots * n_planes * cpp;
-        const long long cap = (long long)sm_count * g_bulk_ctas_per_sm;
+        const long long cap = (long long)sm_count * ctas;
         const int grid = (int)(total < cap ? total : cap);
         copy_bulk_kernel<<<grid, 32, (size_t)g_bulk_chunk * g_bulk_stages, st>>>(
             s.pieces, n_slots, plane0, n_planes, cpp, (unsigned)g_bulk_chunk, g_bulk_stages, s.ctl);
