@@ -69,7 +69,8 @@ typedef enum aaf_status {
     AAF_ERR_CUDA = -8,          /* a CUDA runtime call failed (no usable device, launch error ...)          */
     AAF_ERR_CORRUPT = -9,       /* device found the ring / a reference count inconsistent                   */
     AAF_ERR_TIMEOUT = -10,      /* a bounded device-side wait gave up                                       */
-    AAF_ERR_TOO_MANY = -11      /* batch larger than max_batch                                              */
+    AAF_ERR_TOO_MANY = -11,     /* batch larger than max_batch                                              */
+    AAF_ERR_SCRATCH_LIMIT = -12 /* request larger than the built-in scratch of aaf_kv_materialize_noalloc   */
 } aaf_status;
 
 typedef struct aaf_kv_pool aaf_kv_pool; /* opaque host object */
@@ -214,6 +215,33 @@ int aaf_kv_sync_status(aaf_kv_pool *pool);
 /* Tuning and measurement knobs. */
 int aaf_kv_set_copy_engine(aaf_kv_pool *pool, int engine);  /* AAF_ENGINE_* */
 int aaf_kv_set_timing(aaf_kv_pool *pool, int enable);       /* bracket copy kernels with CUDA events */
+
+/* Gather for callers that cannot allocate -- the paper has no counterpart; this is a library
+ * convenience.  Same result as aaf_kv_materialize (dst[l][kv][t - tok_begin] =
+ * pool[l][table[t / BS]][kv][t % BS] for t in [tok_begin, tok_end)), but it needs no pool object and
+ * no workspace: the caller passes the pool memory and geometry as plain values and the context's
+ * block table as a HOST array (n_table_blocks entries, e.g. from aaf_kv_get_table), and the scratch
+ * the gather needs lives in a fixed array inside the library.  It is meant for callers that must
+ * not call cudaMalloc: a process whose GPU memory is already fully committed to its own pool, a
+ * latency-critical path that cannot take an allocation's device-wide synchronisation, or a plug-in
+ * that is only ever handed pointers.  The call allocates nothing, on the device or in pinned host
+ * memory, and frees nothing.
+ *   - Limit: the token range may touch at most AAF_NOALLOC_MAX_BLOCKS blocks; a larger request
+ *     returns AAF_ERR_SCRATCH_LIMIT and does nothing (split the range).
+ *   - The first call on a device looks up the device address of the built-in array (with the
+ *     calling thread's current device, which must be the one that owns the memory); make that
+ *     first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each
+ *     call clears or overwrites what it reads.  Two calls that overlap on the GPU (different
+ *     streams, or host threads racing) corrupt each other: keep them on one stream or order them.
+ *   - pool_base_dev, dst_dev: device, 16-byte aligned; block_table_host: host, read before return.
+ * Errors: INVALID_ARG (pointers, geometry, range, a table entry outside [0, n_blocks)),
+ * DST_TOO_SMALL, SCRATCH_LIMIT, CUDA. */
+#define AAF_NOALLOC_MAX_BLOCKS 4096
+int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t layer_stride_bytes, int32_t n_layers,
+                               int32_t n_kv_heads, int32_t head_dim, int32_t block_size, int32_t elt_bytes,
+                               int32_t n_blocks, const int32_t *block_table_host, int32_t n_table_blocks,
+                               int64_t tok_begin, int64_t tok_end, void *dst_dev, size_t dst_bytes, void *stream);
 
 const char *aaf_kv_strerror(int status);
 

@@ -18,7 +18,8 @@ AAF_KV_ABI_VERSION = 1
 AAF_OK = 0
 AAF_ERR_INVALID_ARG, AAF_ERR_BAD_CTX, AAF_ERR_OOM_BLOCKS, AAF_ERR_OOM_CTX = -1, -2, -3, -4
 AAF_ERR_TOO_LONG, AAF_ERR_INCOMPAT, AAF_ERR_DST_TOO_SMALL, AAF_ERR_CUDA = -5, -6, -7, -8
-AAF_ERR_CORRUPT, AAF_ERR_TIMEOUT, AAF_ERR_TOO_MANY = -9, -10, -11
+AAF_ERR_CORRUPT, AAF_ERR_TIMEOUT, AAF_ERR_TOO_MANY, AAF_ERR_SCRATCH_LIMIT = -9, -10, -11, -12
+AAF_NOALLOC_MAX_BLOCKS = 4096
 AAF_COMPOSE_SHARE, AAF_COMPOSE_COPY_ALL = 0, 1
 AAF_ENGINE_AUTO, AAF_ENGINE_VEC, AAF_ENGINE_BULK = 0, 1, 2
 AAF_OP_MATERIALIZE, AAF_OP_IMPORT, AAF_OP_APPEND, AAF_OP_COMPOSE, AAF_OP_CLASSES = 0, 1, 2, 3, 4
@@ -78,6 +79,8 @@ SYMBOLS = {
     "aaf_kv_sync_status": (C.c_int, [_vp]),
     "aaf_kv_set_copy_engine": (C.c_int, [_vp, C.c_int]),
     "aaf_kv_set_timing": (C.c_int, [_vp, C.c_int]),
+    "aaf_kv_materialize_noalloc": (C.c_int, [_vp, _sz, _i32, _i32, _i32, _i32, _i32, _i32, _p32, _i32, _i64, _i64, _vp,
+                                             _sz, _vp]),
     "aaf_kv_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -128,6 +131,13 @@ def aaf_kv_pool_stats(pool, out): return _fn("aaf_kv_pool_stats")(pool, out)
 def aaf_kv_sync_status(pool): return _fn("aaf_kv_sync_status")(pool)
 def aaf_kv_set_copy_engine(pool, engine): return _fn("aaf_kv_set_copy_engine")(pool, engine)
 def aaf_kv_set_timing(pool, enable): return _fn("aaf_kv_set_timing")(pool, enable)
+def aaf_kv_materialize_noalloc(pool_base, layer_stride, n_layers, n_kv_heads, head_dim, block_size, elt_bytes, n_blocks,
+                               block_table_host, n_table_blocks, t0, t1, dst, dst_bytes, stream):
+    """Gather without any allocation (see include/aaf_kv.h): for callers that may not call cudaMalloc.
+    block_table_host is a ctypes int32 array / pointer in host memory."""
+    return _fn("aaf_kv_materialize_noalloc")(pool_base, layer_stride, n_layers, n_kv_heads, head_dim, block_size,
+                                             elt_bytes, n_blocks, block_table_host, n_table_blocks, t0, t1, dst,
+                                             dst_bytes, stream)
 def aaf_kv_strerror(status): return _fn("aaf_kv_strerror")(status).decode()
 
 

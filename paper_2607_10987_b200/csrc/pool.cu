@@ -689,6 +689,8 @@ const char *aaf_kv_strerror(int status) {
         case AAF_ERR_CORRUPT: return "device found pool metadata inconsistent";
         case AAF_ERR_TIMEOUT: return "bounded device wait expired";
         case AAF_ERR_TOO_MANY: return "batch exceeds max_batch or the piece capacity";
+        case AAF_ERR_SCRATCH_LIMIT:
+            return "request exceeds the built-in scratch of aaf_kv_materialize_noalloc (AAF_NOALLOC_MAX_BLOCKS blocks)";
         default: return "unknown status";
     }
 }

@@ -73,8 +73,8 @@ def test_create_rejects_bad_arguments_before_touching_a_device():
 
 
 def test_strerror_names_every_status():
-    seen = {binding.aaf_kv_strerror(s) for s in range(0, -12, -1)}
-    assert len(seen) == 12 and "unknown status" not in seen
+    seen = {binding.aaf_kv_strerror(s) for s in range(0, -13, -1)}
+    assert len(seen) == 13 and "unknown status" not in seen
     assert binding.aaf_kv_strerror(-99) == "unknown status"
 
 
