@@ -26,8 +26,12 @@ class OracleBackend:
         if init_fill:
             pv = self.o.pool_view()
             per_layer = g.layer_stride // 2  # elements
+            step = 1 << 24  # elements per chunk: keeps the generator's temporaries small
             for i, l in enumerate(self.layers):
-                pv[i].reshape(-1).view(np.uint16)[:] = fill.fill_np(seed, 0, l * per_layer, per_layer)
+                flat = pv[i].reshape(-1).view(np.uint16)
+                for a in range(0, per_layer, step):
+                    c = min(step, per_layer - a)
+                    flat[a:a + c] = fill.fill_np(seed, 0, l * per_layer + a, c)
 
     def payload(self, seed, stream, n):
         g = self.g

@@ -1,0 +1,74 @@
+"""Parity at the full sizes of the workloads, in the launch configuration the benchmark times.
+
+The GPU library runs the whole geometry; the CPU oracle runs the same operator list on a sample of
+the layers (layers are independent and share block ids), which gives the exact tables, reference
+counts and free list of the full geometry and the exact bytes of the sampled layers: every
+materialised buffer and the final pool image of those layers are compared byte for byte.
+"""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+from tests.test_gpu_parity import lockstep
+from workloads import configs
+from workloads.configs import Geometry
+
+pytestmark = pytest.mark.gpu
+
+
+def _fits(g: Geometry, extra_gib: float) -> bool:
+    free_b, _ = torch.cuda.mem_get_info()
+    return free_b > g.pool_bytes + extra_gib * 2**30
+
+
+@pytest.mark.parametrize("unaligned", [False, True])
+def test_config2_llama8b_full_pool(unaligned):
+    g, seed, ops = configs.config2(unaligned)
+    if not _fits(g, 12):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    gpu, cpu = lockstep(g, seed, ops, layers=[0, g.n_layers - 1])
+    st = gpu.o.stats()
+    assert st["cow_count"] == (16 if unaligned else 0)
+    assert st["live_blocks"] == (512 + 512 + 16 * 32 + (16 if unaligned else 0))
+
+
+def test_config2_single_appends_give_the_same_state():
+    g, seed, ops_b = configs.config2(True)
+    _, _, ops_s = configs.config2(True, batched_append=False)
+    small = Geometry(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, 4096, g.max_ctx,
+                     g.max_blocks_per_ctx)
+    ga, _ = lockstep(small, seed, ops_b, layers=[7])
+    snap_a, img_a = ga.snapshot(), ga.pool_layers([7])
+    del ga
+    gb, _ = lockstep(small, seed, ops_s, layers=[7])
+    assert gb.snapshot() == snap_a
+    assert np.array_equal(gb.pool_layers([7]), img_a)
+
+
+@pytest.mark.parametrize("copy_all", [False, True])
+def test_config3_compose_levels_8b(copy_all):
+    g, seed, ops, lens = configs.config3(configs.LLAMA8B, copy_all=copy_all)
+    if not _fits(g, 16):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    gpu, cpu = lockstep(g, seed, ops, layers=[3, 30])
+    assert gpu.o.ctx_len(gpu.o.live_ctxs()[-1]) == sum(lens)
+
+
+@pytest.mark.parametrize("unaligned", [False, True])
+def test_config4_llama70b(unaligned):
+    g, seed, ops = configs.config4(unaligned)
+    if not _fits(g, 40):
+        pytest.skip("not enough free device memory for the 40 GiB pool plus 10 GiB buffers")
+    gpu, cpu = lockstep(g, seed, ops, layers=[0, 79])
+    assert gpu.o.stats()["cow_count"] == (8 if unaligned else 0)
+
+
+def test_cow_stress_1024_children_8b_rows():
+    g = Geometry(32, 8, 128, 16, 2, 4096, 1100, 1024)
+    ops = configs.cow_stress_ops(context_tokens=8187, n_children=1024)
+    gpu, cpu = lockstep(g, configs.SEED_BASE + 6, ops, layers=[0, 31], max_batch=1024)
+    st = gpu.o.stats()
+    assert st["cow_count"] == 1024
+    assert st["live_blocks"] == 512 + 1024
