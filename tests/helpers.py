@@ -20,6 +20,7 @@ class OracleBackend:
 
     def __init__(self, g: Geometry, seed: int, layers=None, free_order=None, init_fill=True):
         self.g = g
+        self.seed_ = seed
         self.layers = list(range(g.n_layers)) if layers is None else list(layers)
         self.o = paged.PagedOracle(len(self.layers), g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes,
                                    g.n_blocks, g.max_ctx, g.max_blocks_per_ctx, free_order)
@@ -38,6 +39,23 @@ class OracleBackend:
         per_layer = 2 * n * g.row // 2  # elements of one layer of the [L,2,n,H,D] buffer
         parts = [fill.fill_np(seed, stream, l * per_layer, per_layer) for l in self.layers]
         return np.concatenate(parts).view(np.uint8)
+
+    def window(self, op_index, n):
+        """n-token payload read from a window of stream 1 (churn workload): the same elements the GPU
+        backend's window holds, restricted to this oracle's layers."""
+        from workloads.churn import MAX_SEG_TOKENS, WINDOW_SLACK
+
+        g = self.g
+        hd = g.row // 2
+        if getattr(self, "_big", None) is None:
+            total = g.n_layers * 2 * MAX_SEG_TOKENS * hd + WINDOW_SLACK
+            self._big = np.empty(total, dtype=np.uint16)
+            for a in range(0, total, 1 << 24):
+                c = min(1 << 24, total - a)
+                self._big[a:a + c] = fill.fill_np(self.seed_, 1, a, c)
+        o = (op_index * 8) % WINDOW_SLACK
+        per_layer = 2 * n * hd
+        return np.concatenate([self._big[o + l * per_layer: o + (l + 1) * per_layer] for l in self.layers]).view(np.uint8)
 
     def imp(self, buf, n):
         return self.o.imp(buf, n)
@@ -166,55 +184,4 @@ def expected_bytes(seed: int, g: Geometry, tokens, layers=None) -> np.ndarray:
     return out.view(np.uint8).reshape(len(layers), 2, len(tokens), g.row)
 
 
-class GpuBackend:
-    """The CUDA library (through its Python binding) behind the replay-backend interface."""
-
-    def __init__(self, g: Geometry, seed: int, free_order=None, engine: int = 0, init_fill=True, max_batch=0):
-        import torch
-
-        from paper_2607_10987_b200 import KVPool
-
-        self.g, self.torch = g, torch
-        self.o = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, g.n_blocks, g.max_ctx,
-                        g.max_blocks_per_ctx, free_order=free_order, max_batch=max_batch)
-        self.o.set_copy_engine(engine)
-        if init_fill:
-            fill.fill_torch(seed, 0, 0, g.pool_bytes // 2, self.o.device, out=self.o.pool.view(torch.int16))
-        torch.cuda.synchronize()
-
-    def payload(self, seed, stream, n):
-        g = self.g
-        return fill.fill_torch(seed, stream, 0, g.n_layers * 2 * n * g.row // 2, self.o.device).view(self.torch.uint8)
-
-    def imp(self, buf, n):
-        return self.o.imp(buf, n)
-
-    def materialize(self, c, t0, t1):
-        return self.o.materialize(c, t0, t1)
-
-    def fork(self, c, k):
-        return self.o.fork(c, k)
-
-    def append(self, ctxs, n_new, bufs):
-        return self.o.append(ctxs, n_new, bufs)
-
-    def compose(self, ctxs, flags):
-        return self.o.compose(ctxs, flags)
-
-    def evict(self, ctxs):
-        return self.o.evict(ctxs)
-
-    def snapshot(self):
-        return snapshot(self.o)
-
-    def pool_layers(self, layers) -> np.ndarray:
-        """uint8 [len(layers), NB, 2, BS, row] copy of the given layers of the device pool."""
-        g = self.g
-        v = self.o.pool[: g.pool_bytes].view(g.n_layers, g.n_blocks, 2, g.block_size, g.row)
-        return v[list(layers)].cpu().numpy()
-
-    def buf_layers(self, buf, n, layers) -> np.ndarray:
-        """uint8 [len(layers), 2, n, row] copy of the given layers of a device transfer buffer."""
-        g = self.g
-        v = buf[: n * g.bpt].view(g.n_layers, 2, n, g.row)
-        return v[list(layers)].cpu().numpy()
+from paper_2607_10987_b200.replay_backend import GpuBackend  # noqa: E402,F401  (re-exported for the tests)
