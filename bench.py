@@ -192,6 +192,139 @@ def reference_arm(args, w):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------------- other workloads
+def extra_report(args):
+    """Reports for the workloads that are parity cases rather than the headline step: the copy-on-write
+    stress (1024 children of one unaligned context, one batched 1-token append), the composition levels
+    (pairs / quads / all 16) and the churn trace.  One JSON line each, kernel GB/s from the library's
+    CUDA events, bytes from the library's device-side byte counter."""
+    import torch
+
+    from paper_2607_10987_b200 import binding
+    from paper_2607_10987_b200.replay_backend import GpuBackend
+    from workloads import churn
+    from workloads.replay import replay
+
+    binding.load()
+    assert torch.cuda.is_available()
+    dev = torch.device("cuda", 0)
+    peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]) if os.path.exists(
+        os.path.join(ROOT, "MEASURED_PEAKS.json")) else 6650.0
+    out = {"workload": args.workload, "engine": args.engine, "peak_GBps": peak}
+
+    def timed(pool, fn):
+        """runs fn with kernel timing on; returns (wall ms on the stream, per-class kernel ms, bytes one way)"""
+        s0 = pool.stats()
+        pool.set_timing(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        pool.set_timing(False)
+        s1 = pool.stats()
+        dms = {k: s1["copy_ms"][k] - s0["copy_ms"][k] for k in s1["copy_ms"]}
+        return e0.elapsed_time(e1), dms, s1["payload_bytes"] - s0["payload_bytes"]
+
+    if args.workload == "cow":
+        g = configs.Geometry(32, 8, 128, 16, 2, 4096, 1100, 1024)
+        seed = configs.SEED_BASE + 6
+        be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False,
+                        max_batch=1024)
+        T, kids_n = 8187, 1024
+        root_buf = be.payload(seed, 1, T)
+        eight = [be.payload(seed, 2 + i, 1) for i in range(8)]
+        one = [eight[i % 8] for i in range(kids_n)]
+        acc = {"append_ms": 0.0, "append_bytes": 0, "fork_ms": 0.0, "evict_ms": 0.0}
+        for it in range(args.warmup + args.steps):
+            st, root = be.imp(root_buf, T)
+            res = {}
+            ms_f, _, _ = timed(be.o, lambda: res.update(r=be.fork(root, kids_n)))
+            kids = res["r"][1]
+            ms_a, dms, b = timed(be.o, lambda: res.update(a=be.append(kids, [1] * kids_n, one)[0]))
+            assert res["a"] == 0
+            ms_e, _, _ = timed(be.o, lambda: res.update(e=(be.evict(kids)[0], be.evict([root])[0])))
+            assert res["r"][0] == 0 and res["e"] == (0, 0), res
+            if it >= args.warmup:
+                acc["append_ms"] += dms["append"]; acc["append_bytes"] += b
+                acc["fork_ms"] += ms_f; acc["evict_ms"] += ms_e
+        assert be.o.sync_status() == 0 and be.o.stats()["cow_count"] == kids_n * (args.warmup + args.steps)
+        gbps = 2 * acc["append_bytes"] / (acc["append_ms"] * 1e-3) / 1e9
+        out.update({"fork_cow_copy_GBps": gbps, "frac_of_measured_peak": gbps / peak, "frac_of_8TBps": gbps / 8000,
+                    "bytes_moved_per_append_GB": 2 * acc["append_bytes"] / args.steps / 1e9,
+                    "append_kernel_ms": acc["append_ms"] / args.steps, "fork_1024_ms": acc["fork_ms"] / args.steps,
+                    "evict_1024_plus_1_ctx_ms": acc["evict_ms"] / args.steps})
+    elif args.workload == "compose":
+        for copy_all in (False, True):
+            g, seed, ops, lens = configs.config3(configs.LLAMA8B, copy_all=copy_all)
+            be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine,
+                            init_fill=False)
+            levels = {}
+            names = {}
+            imports = [o for o in ops if o["op"] == "import"]
+            composes = [o for o in ops if o["op"] == "compose"]
+            for o in imports:
+                st, c = be.imp(be.payload(seed, o["stream"], o["n"]), o["n"])
+                assert st == 0
+                names[o["out"]] = c
+            for it in range(args.warmup + args.steps):
+                made = []
+                for o in composes:
+                    segs = [names[x] for x in o["segs"]]
+                    res = {}
+                    ms, dms, b = timed(be.o, lambda: res.update(r=be.compose(segs, o["flags"])))
+                    st, c = res["r"]
+                    assert st == 0
+                    names[o["out"]] = c
+                    made.append(c)
+                    if it >= args.warmup:
+                        lv = levels.setdefault(o["level"], {"ms": 0.0, "kernel_ms": 0.0, "bytes": 0, "ops": 0})
+                        lv["ms"] += ms; lv["kernel_ms"] += dms["compose"]; lv["bytes"] += b; lv["ops"] += 1
+                be.evict(made)
+            assert be.o.sync_status() == 0
+            rep = {}
+            for k, lv in levels.items():
+                rep[k] = {"copied_GB_per_op": lv["bytes"] / lv["ops"] / 1e9, "op_ms": lv["ms"] / lv["ops"],
+                          "kernel_GBps": (2 * lv["bytes"] / (lv["kernel_ms"] * 1e-3) / 1e9) if lv["kernel_ms"] else None,
+                          "op_GBps": 2 * lv["bytes"] / (lv["ms"] * 1e-3) / 1e9}
+            out["copy_all" if copy_all else "share"] = rep
+            del be
+            torch.cuda.empty_cache()
+    else:  # churn
+        bs, cap, seed = args.block_size, 32768, configs.SEED_BASE + 5
+        small = lambda nb: configs.Geometry(1, 1, 8, bs, 2, nb, 80, cap // bs)
+        be0 = GpuBackend(small(64 * cap // bs), seed, init_fill=False, staging_tokens=cap)
+        d0 = churn.ChurnDriver(be0, seed, max_ctx_tokens=cap).run(10000)
+        assert all(st == 0 for _, _, st in d0.log)
+        demand = be0.o.stats()["peak_live_blocks"]
+        del be0, d0
+        nb = int(0.75 * demand)
+        g = configs.Geometry(32, 8, 128, bs, 2, nb, 80, cap // bs)
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        if g.pool_bytes + (12 << 30) > free_b:
+            out.update({"skipped": "pool of %.1f GiB does not fit" % (g.pool_bytes / 2**30)})
+        else:
+            be = GpuBackend(g, seed, free_order=configs.free_order(seed, nb), engine=args.engine, init_fill=False,
+                            staging_tokens=cap)
+            be.window(0, 1)
+            d = churn.ChurnDriver(be, seed, max_ctx_tokens=cap)
+            t0 = time.perf_counter()
+            ms, dms, b = timed(be.o, lambda: d.run(10000))
+            wall = time.perf_counter() - t0
+            assert be.o.sync_status() == 0
+            calls = len(d.log)
+            kms = sum(dms.values())
+            out.update({"block_size": bs, "demand_blocks": demand, "n_blocks": nb, "pool_GiB": g.pool_bytes / 2**30,
+                        "library_calls": calls, "calls_by_kind": d.counts,
+                        "oom_answers": sum(1 for _, _, st in d.log if st == churn.OOM_BLOCKS),
+                        "moved_TB": 2 * b / 1e12, "stream_ms": ms, "wall_s": wall, "ops_per_s": 10000 / wall,
+                        "calls_per_s": calls / wall, "GBps_whole_trace": 2 * b / wall / 1e9,
+                        "copy_kernel_GBps": 2 * b / (kms * 1e-3) / 1e9, "peak_live_blocks": be.o.stats()["peak_live_blocks"],
+                        "cow_count": be.o.stats()["cow_count"]})
+    print(json.dumps(out), flush=True)
+
+
 # ------------------------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -199,11 +332,14 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn"])
+    ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST, 2 cp.async.bulk")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    if args.workload in ("cow", "compose", "churn"):
+        return extra_report(args)
     w = workload(args.workload)
     if args.impl == "reference":
         reference_arm(args, w)
@@ -295,16 +431,24 @@ def main():
         d_agents = torch.empty(agents * n_new * g.bpt, dtype=torch.uint8, device=dev)
         views = [d_agents[i * n_new * g.bpt:(i + 1) * n_new * g.bpt] for i in range(agents)]
 
+        side = torch.cuda.Stream(dev)  # prefetches the continuation tokens while the transfer buffer goes back
+        fetched = torch.cuda.Event()
+
         def e2e_step():
+            main = torch.cuda.current_stream(dev)
             st, root = pool.import_host(h_root, T, d_root)  # H2D + scatter
             assert st == 0, st
-            st = pool.materialize_host(root, 0, T, h_out, staging)  # gather + D2H
+            side.wait_stream(main)  # d_agents is free once the previous step's append has run
+            with torch.cuda.stream(side):
+                d_agents.copy_(h_agents, non_blocking=True)  # H2D of the continuation tokens
+                fetched.record(side)
+            st = pool.materialize_host(root, 0, T, h_out, staging)  # gather + D2H (overlaps the H2D above)
             assert st == 0, st
             st, recv = pool.imp(staging, T)
             assert st == 0, st
             st, kids = pool.fork(recv, agents)
             assert st == 0, st
-            d_agents.copy_(h_agents, non_blocking=True)  # H2D of the continuation tokens
+            main.wait_event(fetched)
             st, _ = pool.append(kids, [n_new] * agents, views)
             assert st == 0, st
             st, merged = pool.compose(kids[:2], 0)

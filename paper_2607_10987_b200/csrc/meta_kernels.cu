@@ -51,6 +51,21 @@ __device__ __forceinline__ void claim_block(const DevState &s, int b, int NB) {
     s.refcount[b] = 1;
 }
 
+// Argument records arrive in pinned host memory that the kernel reads over PCIe; every such read costs
+// a bus round trip and is not cached, so a kernel that searches its records stages them first: one
+// coalesced pass into shared memory (when they fit), then all further reads are on-chip.
+template <typename T>
+__device__ __forceinline__ const T *stage_args(const T *src, int count, T *smem_buf, int cap) {
+    static_assert(sizeof(T) % 4 == 0, "records are copied as 32-bit words");
+    if (count > cap) return src;
+    const int words = count * (int)(sizeof(T) / 4);
+    const int *s32 = reinterpret_cast<const int *>(src);
+    int *d32 = reinterpret_cast<int *>(smem_buf);
+    for (int i = threadIdx.x; i < words; i += blockDim.x) d32[i] = s32[i];
+    __syncthreads();
+    return smem_buf;
+}
+
 // CTA-wide exclusive prefix sum of one int per thread (warp shuffles + one shared array).
 // Returns the exclusive prefix of `v`; *total receives the CTA's sum.
 __device__ __forceinline__ int block_exclusive_scan(int v, int *total) {
@@ -134,7 +149,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevSt
 // ------------------------------------------------------------------------------------------
 // fork: k table copies, refcount += k per parent entry
 __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int parent, int nblk, int k,
-                                                   const int *__restrict__ children) {
+                                                   const int *__restrict__ children_host) {
+    __shared__ int sh_children[1024];
+    const int *children = stage_args(children_host, k, sh_children, 1024);
     const int *pt = s.tables + (long long)parent * g.max_blk;
     const long long total = (long long)nblk * k;
     for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
@@ -157,8 +174,10 @@ __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int paren
 //
 // scratch layout (ints): tailb[n] | need[n] | alloc_off[n]
 __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevState s,
-                                                                   const AppendEntry *__restrict__ ent, int n,
+                                                                   const AppendEntry *__restrict__ ent_host, int n,
                                                                    int total_slots, int max_batch, int dry_run) {
+    __shared__ AppendEntry sh_ent[768];
+    const AppendEntry *ent = stage_args(ent_host, n, sh_ent, 768);
     int *tailb = s.scratch;
     int *need = s.scratch + max_batch;
     int *alloc_off = s.scratch + 2 * max_batch;
@@ -277,9 +296,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 //   copy segment  : item w -> destination block nblk(off)-(off%BS>0) + w, which receives tokens
 //                   from at most two source blocks (two piece slots per item)
 __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
-                                                                    const ComposeSeg *__restrict__ segs, int m,
+                                                                    const ComposeSeg *__restrict__ segs_host, int m,
                                                                     int total_work, int total_fresh, int total_slots,
                                                                     int out_ctx) {
+    __shared__ ComposeSeg sh_segs[512];
+    const ComposeSeg *segs = stage_args(segs_host, m, sh_segs, 512);
     const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
     const bool ok = (tail - head0) >= (unsigned long long)total_fresh;
     int *out = s.tables + (long long)out_ctx * g.max_blk;
@@ -365,9 +386,12 @@ __device__ __forceinline__ int evict_entry_block(const Geom &g, const DevState &
     return s.tables[(long long)ctx[lo] * g.max_blk + (e - ent_off[lo])];
 }
 
-__global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a) {
-    const int n = a->n, total = a->total;
-    const int *ctx = reinterpret_cast<const int *>(a + 1);
+constexpr int EVICT_STAGE = 2048;  // ints: ctx[n] followed by ent_off[n + 1]
+
+__global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a,
+                                                            int n, int total) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
     const int *ent_off = ctx + n;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
         const int b = evict_entry_block(g, s, ctx, ent_off, n, e);
@@ -377,9 +401,10 @@ __global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, 
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
-                                                                  const EvictArgs *__restrict__ a) {
-    const int n = a->n, total = a->total;
-    const int *ctx = reinterpret_cast<const int *>(a + 1);
+                                                                  const EvictArgs *__restrict__ a, int n,
+                                                                  int total) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
     const int *ent_off = ctx + n;
     const unsigned long long tail0 = s.ctl->tail;
     int carry = 0;
@@ -442,11 +467,10 @@ cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeS
 }
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
                          cudaStream_t st) {
-    (void)n;
-    evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev);
+    evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev, n, total);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev);
+    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total);
     return cudaGetLastError();
 }
 

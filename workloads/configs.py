@@ -70,7 +70,7 @@ class Geometry:
 
 TINY = Geometry(2, 2, 64, 16, 2, 256, 16, 128)
 LLAMA8B = Geometry(32, 8, 128, 16, 2, 32768, 64, 4096)
-LLAMA70B = Geometry(80, 8, 128, 16, 2, 8192, 32, 4096)
+LLAMA70B = Geometry(80, 8, 128, 16, 2, 8192, 32, 8192)
 
 
 def free_order(seed: int, n_blocks: int) -> np.ndarray:
