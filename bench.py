@@ -44,7 +44,7 @@ UNIT = "GB/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per algorithmic byte for the copy kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
-TRAFFIC_PER_ALGORITHMIC_BYTE = None
+TRAFFIC_PER_ALGORITHMIC_BYTE = 0.91  # profiles/copy_vec_kernel_8b-small_ncu_full.md: (267.8 + 219.6) / (2 x 267.8) MB
 
 
 def workload(name: str):
@@ -334,7 +334,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn"])
     ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
-    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST, 2 cp.async.bulk")
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST per CTA, 2 cp.async.bulk, 3 vector LD/ST per warp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()

@@ -112,6 +112,7 @@ typedef struct aaf_kv_xfer_desc {
 #define AAF_ENGINE_AUTO 0        /* the library picks                                                     */
 #define AAF_ENGINE_VEC 1         /* 16-byte vector loads/stores through registers                         */
 #define AAF_ENGINE_BULK 2        /* cp.async.bulk global->shared->global with mbarrier completion         */
+#define AAF_ENGINE_WARP 3        /* 16-byte vector copies scheduled per warp (best for small / ragged pieces) */
 
 /* operator classes that move payload (index into the per-class arrays of aaf_kv_stats) */
 #define AAF_OP_MATERIALIZE 0

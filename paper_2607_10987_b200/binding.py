@@ -21,7 +21,7 @@ AAF_ERR_TOO_LONG, AAF_ERR_INCOMPAT, AAF_ERR_DST_TOO_SMALL, AAF_ERR_CUDA = -5, -6
 AAF_ERR_CORRUPT, AAF_ERR_TIMEOUT, AAF_ERR_TOO_MANY, AAF_ERR_SCRATCH_LIMIT = -9, -10, -11, -12
 AAF_NOALLOC_MAX_BLOCKS = 4096
 AAF_COMPOSE_SHARE, AAF_COMPOSE_COPY_ALL = 0, 1
-AAF_ENGINE_AUTO, AAF_ENGINE_VEC, AAF_ENGINE_BULK = 0, 1, 2
+AAF_ENGINE_AUTO, AAF_ENGINE_VEC, AAF_ENGINE_BULK, AAF_ENGINE_WARP = 0, 1, 2, 3
 AAF_OP_MATERIALIZE, AAF_OP_IMPORT, AAF_OP_APPEND, AAF_OP_COMPOSE, AAF_OP_CLASSES = 0, 1, 2, 3, 4
 OP_NAMES = ("materialize", "import", "append", "compose")
 

@@ -91,8 +91,16 @@ cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeS
                                 int total_fresh, int total_slots, int out_ctx, cudaStream_t st);
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
                          cudaStream_t st);
-cudaError_t launch_copy(int engine, const Geom &g, const DevState &s, int n_slots, int plane0, int n_planes,
-                        int sm_count, cudaStream_t st);
-cudaError_t copy_engine_init(int device);
+// launch shapes of the copy engines for one pool geometry (see copy_tuning_init)
+struct CopyTuning {
+    int bulk_chunk, bulk_stages, bulk_ctas, bulk_l2;
+    int vec_unroll, vec_ctas;
+    int warp_unroll, warp_ctas;
+    int auto_engine;               // 0 = choose per launch, else forced engine
+    long long auto_bulk_min_piece; // AUTO: mean piece size from which the bulk engine is used
+};
+cudaError_t copy_tuning_init(long long run, CopyTuning *t);
+cudaError_t launch_copy(int engine, const CopyTuning &t, const Geom &g, const DevState &s, int n_slots, int plane0,
+                        int n_planes, long long avg_piece_bytes, int sm_count, cudaStream_t st);
 
 }  // namespace aafkv

@@ -85,6 +85,50 @@ __global__ void __launch_bounds__(VEC_THREADS) copy_vec_kernel(const Piece *__re
 }
 
 // ------------------------------------------------------------------------------------------
+// WARP engine: the same 16-byte streaming copies, but the unit of work is a warp, not a CTA.  A warp
+// takes 32 consecutive units, decodes all of them at once (one unit per lane, so the descriptor
+// fetches overlap and empty units cost nothing further), then moves them one after the other with
+// all 32 lanes.  Small and ragged pieces (copy-on-write tails, single-token appends, the two
+// part-blocks of a shifted compose) no longer leave most of a CTA idle or serialise on descriptor
+// latency; full runs are split into 32*U*16-byte chunks handled by neighbouring warps.
+template <int UNROLL>
+__global__ void __launch_bounds__(VEC_THREADS) copy_warp_kernel(const Piece *__restrict__ pieces, int n_slots,
+                                                                int plane0, int n_planes, int cpp) {
+    constexpr unsigned CHUNK = 32 * UNROLL * 16;
+    constexpr unsigned FULL = 0xffffffffu;
+    const long long total = (long long)n_slots * n_planes * cpp;
+    const int lane = threadIdx.x & 31;
+    const long long warps = (long long)gridDim.x * (VEC_THREADS / 32);
+    const long long gw = (long long)blockIdx.x * (VEC_THREADS / 32) + (threadIdx.x >> 5);
+    for (long long base = gw * 32; base < total; base += warps * 32) {
+        Unit mine;
+        mine.src = nullptr; mine.dst = nullptr; mine.nbytes = 0;
+        if (base + lane < total) mine = decode_unit(pieces, base + lane, n_slots, plane0, cpp, CHUNK);
+        unsigned todo = __ballot_sync(FULL, mine.nbytes != 0);
+        while (todo) {
+            const int j = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint4 *__restrict__ s4 = reinterpret_cast<const uint4 *>(
+                __shfl_sync(FULL, reinterpret_cast<unsigned long long>(mine.src), j));
+            uint4 *__restrict__ d4 =
+                reinterpret_cast<uint4 *>(__shfl_sync(FULL, reinterpret_cast<unsigned long long>(mine.dst), j));
+            const unsigned nvec = __shfl_sync(FULL, mine.nbytes, j) >> 4;
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k) {
+                const unsigned i = lane + k * 32;
+                if (i < nvec) v[k] = __ldcs(s4 + i);
+            }
+#pragma unroll
+            for (int k = 0; k < UNROLL; ++k) {
+                const unsigned i = lane + k * 32;
+                if (i < nvec) __stcs(d4 + i, v[k]);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // BULK engine
 constexpr int BULK_MAX_STAGES = 8;
 constexpr long long BULK_WAIT_CYCLES = 1ll << 32;  // about two seconds of SM clock
@@ -117,15 +161,36 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity)
     }
     return true;
 }
-__device__ __forceinline__ void bulk_g2s(unsigned smem_dst, const void *gsrc, unsigned bytes, unsigned bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_dst),
-                 "l"(gsrc), "r"(bytes), "r"(bar)
-                 : "memory");
+// L2 policy for data that is touched once: mark the lines evict-first so that the stream does not push
+// other tenants' data out of the 126 MB L2
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
-__device__ __forceinline__ void bulk_s2g(void *gdst, unsigned smem_src, unsigned bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
-                 : "memory");
+__device__ __forceinline__ void bulk_g2s(unsigned smem_dst, const void *gsrc, unsigned bytes, unsigned bar,
+                                         unsigned long long pol, bool hint) {
+    if (hint)
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::
+                "r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar), "l"(pol)
+            : "memory");
+    else
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_dst),
+                     "l"(gsrc), "r"(bytes), "r"(bar)
+                     : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *gdst, unsigned smem_src, unsigned bytes, unsigned long long pol,
+                                         bool hint) {
+    if (hint)
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
+                     "r"(smem_src), "r"(bytes), "l"(pol)
+                     : "memory");
+    else
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src),
+                     "r"(bytes)
+                     : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
@@ -133,13 +198,15 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__ pieces, int n_slots, int plane0,
                                                        int n_planes, int cpp, unsigned chunk, int stages,
-                                                       DevCtl *ctl) {
+                                                       int l2_hints, DevCtl *ctl) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long bars[BULK_MAX_STAGES];
     if (threadIdx.x != 0) return;
 
     const long long total = (long long)n_slots * n_planes * cpp;
     const unsigned smem0 = smem_u32(smem);
+    const unsigned long long pol = l2_evict_first_policy();
+    const bool hint_ld = (l2_hints & 1) != 0, hint_st = (l2_hints & 2) != 0;
     for (int s = 0; s < stages; ++s) mbar_init(smem_u32(&bars[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -160,7 +227,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
             const int s = k_load % stages;
             const unsigned bar = smem_u32(&bars[s]);
             mbar_expect_tx(bar, un.nbytes);
-            bulk_g2s(smem0 + (unsigned)s * chunk, un.src, un.nbytes, bar);
+            bulk_g2s(smem0 + (unsigned)s * chunk, un.src, un.nbytes, bar, pol, hint_ld);
             dstq[s] = un.dst;
             nbq[s] = un.nbytes;
             ++k_load;
@@ -178,7 +245,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
             timed_out = true;
             break;
         }
-        bulk_s2g(dstq[s], smem0 + (unsigned)s * chunk, nbq[s]);
+        bulk_s2g(dstq[s], smem0 + (unsigned)s * chunk, nbq[s], pol, hint_st);
         bulk_commit();
         ++k_store;
         // the stage of the store before this one is the next load target: wait until that store has
@@ -198,13 +265,6 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
 // ------------------------------------------------------------------------------------------
 // host side
 
-static int g_bulk_chunk = 16384;
-static int g_bulk_stages = 4;
-static int g_bulk_ctas_per_sm = 3;
-static int g_vec_unroll = 4;
-static int g_vec_ctas_per_sm = 8;  // upper limit; the launch uses min(this, resident CTAs per SM)
-static int g_auto_engine = AAF_ENGINE_VEC;
-
 static int env_int(const char *name, int dflt, int lo, int hi) {
     const char *v = getenv(name);
     if (!v || !*v) return dflt;
@@ -213,66 +273,101 @@ static int env_int(const char *name, int dflt, int lo, int hi) {
     return (int)x;
 }
 
-// Reads the tuning knobs (environment, for experiments) and opts the bulk kernel in to the shared
-// memory it needs.  Called once per pool creation with the pool's device current.
-cudaError_t copy_engine_init(int device) {
-    (void)device;
-    g_bulk_chunk = env_int("AAFKV_BULK_CHUNK", g_bulk_chunk, 1024, 65536) & ~15;
-    g_bulk_stages = env_int("AAFKV_BULK_STAGES", g_bulk_stages, 2, BULK_MAX_STAGES);
-    g_bulk_ctas_per_sm = env_int("AAFKV_BULK_CTAS", g_bulk_ctas_per_sm, 1, 16);
-    g_vec_unroll = env_int("AAFKV_VEC_UNROLL", g_vec_unroll, 1, 8);
-    g_vec_ctas_per_sm = env_int("AAFKV_VEC_CTAS", g_vec_ctas_per_sm, 1, 8);
-    g_auto_engine = env_int("AAFKV_ENGINE", g_auto_engine, 1, 2);
-    while ((long long)g_bulk_chunk * g_bulk_stages > 220 * 1024) --g_bulk_stages;
-    return cudaFuncSetAttribute(copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                g_bulk_chunk * g_bulk_stages);
-}
-
-// resident CTAs per SM of a kernel, capped by the knob: the persistent grid must fit in ONE wave,
+// resident CTAs per SM of a kernel, capped by `limit`: the persistent grid must fit in ONE wave,
 // otherwise the CTAs of the second wave start when the first ones are done and the tail doubles
 template <typename K>
-static int resident_ctas(K kernel, int threads, size_t dyn_smem, int knob) {
+static int resident_ctas(K kernel, int threads, size_t dyn_smem, int limit) {
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, threads, dyn_smem) != cudaSuccess || occ < 1) {
         cudaGetLastError();
         occ = 1;
     }
-    return occ < knob ? occ : knob;
+    return occ < limit ? occ : limit;
+}
+
+// Picks the launch shapes for a pool geometry (run = bytes of one block, one layer, K or V).
+// Defaults come from measurements on B200 with 2 KiB rows; every knob can be overridden through the
+// environment for experiments (AAFKV_ENGINE, AAFKV_BULK_CHUNK / _STAGES / _CTAS / _L2, AAFKV_VEC_UNROLL /
+// _CTAS, AAFKV_WARP_UNROLL).  Called with the pool's device current; allocates nothing.
+cudaError_t copy_tuning_init(long long run, CopyTuning *t) {
+    long long chunk = run < 32768 ? ((run + 15) / 16) * 16 : 32768;
+    if (chunk < 1024) chunk = 1024;
+    t->bulk_chunk = env_int("AAFKV_BULK_CHUNK", (int)chunk, 1024, 65536) & ~15;
+    t->bulk_stages = env_int("AAFKV_BULK_STAGES", 3, 2, BULK_MAX_STAGES);
+    while ((long long)t->bulk_chunk * t->bulk_stages > 220 * 1024) --t->bulk_stages;
+    int ctas = (int)(196608 / ((long long)t->bulk_chunk * t->bulk_stages));  // fill about 192 KiB per SM
+    if (ctas < 1) ctas = 1;
+    if (ctas > 8) ctas = 8;
+    t->bulk_ctas = env_int("AAFKV_BULK_CTAS", ctas, 1, 16);
+    t->bulk_l2 = env_int("AAFKV_BULK_L2", 3, 0, 3);
+    t->vec_unroll = env_int("AAFKV_VEC_UNROLL", 4, 1, 8);
+    if (t->vec_unroll == 3 || (t->vec_unroll > 4 && t->vec_unroll < 8)) t->vec_unroll = 4;
+    t->warp_unroll = env_int("AAFKV_WARP_UNROLL", 8, 4, 8) == 4 ? 4 : 8;
+    t->auto_engine = env_int("AAFKV_ENGINE", 0, 0, 3);
+    t->auto_bulk_min_piece = (long long)t->bulk_chunk * 7 / 16;  // 14 KiB with 32 KiB chunks
+    const cudaError_t e = cudaFuncSetAttribute(copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               220 * 1024);
+    if (e != cudaSuccess) return e;
+    t->bulk_ctas = resident_ctas(copy_bulk_kernel, 32, (size_t)t->bulk_chunk * t->bulk_stages, t->bulk_ctas);
+    const int vlim = env_int("AAFKV_VEC_CTAS", 8, 1, 8);
+    switch (t->vec_unroll) {
+        case 1: t->vec_ctas = resident_ctas(copy_vec_kernel<1>, VEC_THREADS, 0, vlim); break;
+        case 2: t->vec_ctas = resident_ctas(copy_vec_kernel<2>, VEC_THREADS, 0, vlim); break;
+        case 8: t->vec_ctas = resident_ctas(copy_vec_kernel<8>, VEC_THREADS, 0, vlim); break;
+        default: t->vec_ctas = resident_ctas(copy_vec_kernel<4>, VEC_THREADS, 0, vlim); break;
+    }
+    t->warp_ctas = t->warp_unroll == 4 ? resident_ctas(copy_warp_kernel<4>, VEC_THREADS, 0, 8)
+                                       : resident_ctas(copy_warp_kernel<8>, VEC_THREADS, 0, 8);
+    return cudaSuccess;
 }
 
 template <int UNROLL>
-static void launch_vec(const DevState &s, int n_slots, int plane0, int n_planes, long long run, int sm_count,
-                       cudaStream_t st) {
+static void launch_vec(const CopyTuning &t, const DevState &s, int n_slots, int plane0, int n_planes, long long run,
+                       int sm_count, cudaStream_t st) {
     constexpr long long CHUNK = (long long)VEC_THREADS * UNROLL * 16;
-    static int ctas = 0;  // per template instance; the knobs are fixed after the first pool creation
-    if (ctas == 0) ctas = resident_ctas(copy_vec_kernel<UNROLL>, VEC_THREADS, 0, g_vec_ctas_per_sm);
     const int cpp = (int)((run + CHUNK - 1) / CHUNK);
     const long long total = (long long)n_slots * n_planes * cpp;
-    const long long cap = (long long)sm_count * ctas;
+    const long long cap = (long long)sm_count * t.vec_ctas;
     const int grid = (int)(total < cap ? total : cap);
     copy_vec_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp);
 }
 
-cudaError_t launch_copy(int engine, const Geom &g, const DevState &s, int n_slots, int plane0, int n_planes,
+template <int UNROLL>
+static void launch_warp(const CopyTuning &t, const DevState &s, int n_slots, int plane0, int n_planes, long long run,
                         int sm_count, cudaStream_t st) {
+    constexpr long long CHUNK = 32ll * UNROLL * 16;
+    const int cpp = (int)((run + CHUNK - 1) / CHUNK);
+    const long long total = (long long)n_slots * n_planes * cpp;
+    const long long need = (total + 255) / 256;  // CTAs needed if every warp takes one round of 32 units
+    const long long cap = (long long)sm_count * t.warp_ctas;
+    const int grid = (int)(need < cap ? (need < 1 ? 1 : need) : cap);
+    copy_warp_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp);
+}
+
+// AUTO: pieces of about a run or more -> the bulk engine (fastest, and it leaves the SMs idle);
+// small or ragged pieces -> the warp engine (many independent small copies in flight).
+cudaError_t launch_copy(int engine, const CopyTuning &t, const Geom &g, const DevState &s, int n_slots, int plane0,
+                        int n_planes, long long avg_piece_bytes, int sm_count, cudaStream_t st) {
     if (n_slots <= 0 || n_planes <= 0) return cudaSuccess;
-    if (engine == AAF_ENGINE_AUTO) engine = g_auto_engine;
+    if (engine == AAF_ENGINE_AUTO) engine = t.auto_engine;
+    if (engine == AAF_ENGINE_AUTO)
+        engine = avg_piece_bytes >= t.auto_bulk_min_piece ? AAF_ENGINE_BULK : AAF_ENGINE_WARP;
     if (engine == AAF_ENGINE_BULK) {
-        static int ctas = 0;
-        if (ctas == 0)
-            ctas = resident_ctas(copy_bulk_kernel, 32, (size_t)g_bulk_chunk * g_bulk_stages, g_bulk_ctas_per_sm);
-        const int cpp = (int)((g.run + g_bulk_chunk - 1) / g_bulk_chunk);
+        const int cpp = (int)((g.run + t.bulk_chunk - 1) / t.bulk_chunk);
         const long long total = (long long)n_slots * n_planes * cpp;
-        const long long cap = (long long)sm_count * ctas;
+        const long long cap = (long long)sm_count * t.bulk_ctas;
         const int grid = (int)(total < cap ? total : cap);
-        copy_bulk_kernel<<<grid, 32, (size_t)g_bulk_chunk * g_bulk_stages, st>>>(
-            s.pieces, n_slots, plane0, n_planes, cpp, (unsigned)g_bulk_chunk, g_bulk_stages, s.ctl);
+        copy_bulk_kernel<<<grid, 32, (size_t)t.bulk_chunk * t.bulk_stages, st>>>(
+            s.pieces, n_slots, plane0, n_planes, cpp, (unsigned)t.bulk_chunk, t.bulk_stages, t.bulk_l2, s.ctl);
+    } else if (engine == AAF_ENGINE_WARP) {
+        if (t.warp_unroll == 4) launch_warp<4>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st);
+        else launch_warp<8>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st);
     } else {
-        switch (g_vec_unroll) {
-            case 1: launch_vec<1>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
-            case 2: launch_vec<2>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
-            case 8: launch_vec<8>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
-            default: launch_vec<4>(s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+        switch (t.vec_unroll) {
+            case 1: launch_vec<1>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            case 2: launch_vec<2>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            case 8: launch_vec<8>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
+            default: launch_vec<4>(t, s, n_slots, plane0, n_planes, g.run, sm_count, st); break;
         }
     }
     return cudaGetLastError();

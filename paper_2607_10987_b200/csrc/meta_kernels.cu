@@ -400,6 +400,8 @@ __global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, 
     }
 }
 
+constexpr int EVICT_ITEMS = 8;  // consecutive flattened entries per thread and pass
+
 __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
                                                                   const EvictArgs *__restrict__ a, int n,
                                                                   int total) {
@@ -408,19 +410,54 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevSta
     const int *ent_off = ctx + n;
     const unsigned long long tail0 = s.ctl->tail;
     int carry = 0;
-    for (int base = 0; base < total; base += blockDim.x) {
-        const int e = base + threadIdx.x;
-        int b = -1, flag = 0;
-        if (e < total) {
-            b = evict_entry_block(g, s, ctx, ent_off, n, e);
-            flag = (s.refcount[b] == 0 && s.last_pos[b] == e);
+    for (int base = 0; base < total; base += PLAN_THREADS * EVICT_ITEMS) {
+        const int e0 = base + threadIdx.x * EVICT_ITEMS;
+        int blk[EVICT_ITEMS];
+        // locate the first entry once, then walk (context, position) forward: all table reads are independent
+        int ci = 0;
+        if (e0 < total) {
+            int lo = 0, hi = n - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (ent_off[mid] <= e0) lo = mid; else hi = mid - 1;
+            }
+            ci = lo;
+        }
+#pragma unroll
+        for (int k = 0; k < EVICT_ITEMS; ++k) {
+            const int e = e0 + k;
+            blk[k] = -1;
+            if (e < total) {
+                while (e >= ent_off[ci + 1]) ++ci;
+                blk[k] = s.tables[(long long)ctx[ci] * g.max_blk + (e - ent_off[ci])];
+            }
+        }
+        int rc[EVICT_ITEMS], lp[EVICT_ITEMS];
+#pragma unroll
+        for (int k = 0; k < EVICT_ITEMS; ++k) {
+            rc[k] = blk[k] >= 0 ? s.refcount[blk[k]] : 1;
+            lp[k] = blk[k] >= 0 ? s.last_pos[blk[k]] : -1;
+        }
+        int cnt = 0;
+        unsigned flags = 0;
+#pragma unroll
+        for (int k = 0; k < EVICT_ITEMS; ++k) {
+            const bool f = blk[k] >= 0 && rc[k] == 0 && lp[k] == e0 + k;
+            flags |= (f ? 1u : 0u) << k;
+            cnt += f;
         }
         int tot;
-        const int ex = block_exclusive_scan(flag, &tot);
-        if (flag) s.ring[(tail0 + (unsigned long long)(carry + ex)) % (unsigned long long)g.NB] = b;
+        int pos = carry + block_exclusive_scan(cnt, &tot);
+#pragma unroll
+        for (int k = 0; k < EVICT_ITEMS; ++k)
+            if (flags & (1u << k)) {
+                s.ring[(tail0 + (unsigned long long)pos) % (unsigned long long)g.NB] = blk[k];
+                ++pos;
+            }
         carry += tot;
     }
     __syncthreads();
+    // every flag has been taken: clear the scratch marks of the touched blocks
     for (int e = threadIdx.x; e < total; e += blockDim.x)
         s.last_pos[evict_entry_block(g, s, ctx, ent_off, n, e)] = -1;
     if (threadIdx.x == 0) {

@@ -35,6 +35,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocS
 constexpr int MAX_DEVICES = 64;
 NoAllocScratch *g_scratch_ptr[MAX_DEVICES] = {};  // device address of the array, per device
 int g_sm_count[MAX_DEVICES] = {};
+CopyTuning g_tuning[MAX_DEVICES] = {};     // launch shapes of the copy engine, per device
 
 // first call on a device: resolve the array's device address with that device current
 int setup_device(int dev) {
@@ -46,6 +47,10 @@ int setup_device(int dev) {
     }
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        cudaGetLastError();
+        return AAF_ERR_CUDA;
+    }
+    if (copy_tuning_init(32768, &g_tuning[dev]) != cudaSuccess) {  // occupancy queries only, no allocation
         cudaGetLastError();
         return AAF_ERR_CUDA;
     }
@@ -106,7 +111,8 @@ extern "C" int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t laye
     s.pieces = sc->pieces;
     if (launch_plan_materialize(g, s, 0, tok_begin, tok_end, static_cast<char *>(dst_dev), st) != cudaSuccess)
         return AAF_ERR_CUDA;
-    if (launch_copy(AAF_ENGINE_VEC, g, s, (int)nb, 0, 2 * n_layers, g_sm_count[dev], st) != cudaSuccess)
+    if (launch_copy(AAF_ENGINE_VEC, g_tuning[dev], g, s, (int)nb, 0, 2 * n_layers, run, g_sm_count[dev], st) !=
+        cudaSuccess)
         return AAF_ERR_CUDA;
     return AAF_OK;
 }

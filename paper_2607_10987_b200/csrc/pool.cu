@@ -82,6 +82,7 @@ struct aaf_kv_pool {
     DevState s;
     Layout lay;
     int device = 0, sm_count = 148;
+    CopyTuning tuning{};
     std::vector<long long> len;  // tokens per handle, -1 = free
     int live_ctx = 0;
     long long free_lb = 0;       // guaranteed lower bound of the device's free-block count
@@ -175,7 +176,9 @@ void drain_timing(aaf_kv_pool *p) {
 }
 
 // copy-engine launch for one operator class over planes [plane0, plane0 + n_planes)
-int run_copy(aaf_kv_pool *p, int cls, int n_slots, int plane0, int n_planes, cudaStream_t st) {
+int run_copy(aaf_kv_pool *p, int cls, int n_slots, long long payload_tokens, cudaStream_t st) {
+    const int plane0 = 0, n_planes = 2 * p->g.L;
+    const long long avg_piece = n_slots > 0 ? payload_tokens * p->g.row / n_slots : 0;
     if (n_slots <= 0) return AAF_OK;
     TimedLaunch t{};
     if (p->timing) {
@@ -184,7 +187,7 @@ int run_copy(aaf_kv_pool *p, int cls, int n_slots, int plane0, int n_planes, cud
         t.cls = cls;
         cudaEventRecord(t.start, st);
     }
-    const cudaError_t e = launch_copy(p->engine, p->g, p->s, n_slots, plane0, n_planes, p->sm_count, st);
+    const cudaError_t e = launch_copy(p->engine, p->tuning, p->g, p->s, n_slots, plane0, n_planes, avg_piece, p->sm_count, st);
     if (p->timing) {
         cudaEventRecord(t.stop, st);
         p->pending.push_back(t);
@@ -219,7 +222,7 @@ int materialize_impl(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void
         return AAF_ERR_CUDA;
     p->meta_launches += 1;
     const int n_slots = (int)((t1 - 1) / p->g.BS - t0 / p->g.BS + 1);
-    const int rc = run_copy(p, AAF_OP_MATERIALIZE, n_slots, 0, 2 * p->g.L, st);
+    const int rc = run_copy(p, AAF_OP_MATERIALIZE, n_slots, n, st);
     if (rc == AAF_OK && out_desc) fill_desc(p, out_desc, t0, n);
     return rc;
 }
@@ -249,7 +252,7 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
     p->len[c] = n;
     p->live_ctx += 1;
     *out_ctx = c;
-    return run_copy(p, AAF_OP_IMPORT, (int)nb, 0, 2 * p->g.L, st);
+    return run_copy(p, AAF_OP_IMPORT, (int)nb, n, st);
 }
 
 }  // namespace
@@ -313,7 +316,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     p->free_lb = desc->n_blocks;
 
     bool ok = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) == cudaSuccess;
-    ok = ok && copy_engine_init(p->device) == cudaSuccess;
+    ok = ok && copy_tuning_init(p->g.run, &p->tuning) == cudaSuccess;
     p->slot_bytes = align_up(48 * (size_t)lay.max_batch + 256, 256);
     ok = ok && cudaHostAlloc(reinterpret_cast<void **>(&p->args), p->slot_bytes * ARG_SLOTS, cudaHostAllocMapped) ==
                    cudaSuccess;
@@ -434,10 +437,11 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
         if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AAF_ERR_INVALID_ARG;
     }
     const int BS = p->g.BS;
-    long long worst = 0, slots = 0;
+    long long worst = 0, slots = 0, append_tokens = 0;  // append_tokens: new tokens plus the copy-on-write worst case
     for (int i = 0; i < n; ++i) {
         const long long T = p->len[ctxs[i]];
         if (nblk_of(p, T + n_new[i]) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+        append_tokens += n_new[i] + T % BS;
         worst += (T % BS ? 1 : 0) + nblk_of(p, T + n_new[i]) - nblk_of(p, T);
         slots += 1 + nblk_of(p, T + n_new[i]) - T / BS;
     }
@@ -485,7 +489,7 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
     p->meta_launches += 1;
     p->free_lb -= charge;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] += n_new[i];
-    return run_copy(p, AAF_OP_APPEND, (int)slots, 0, 2 * p->g.L, st);
+    return run_copy(p, AAF_OP_APPEND, (int)slots, append_tokens, st);
 }
 
 int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
@@ -498,7 +502,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     const int BS = p->g.BS;
     // everything but the block ids follows from the lengths
     std::vector<ComposeSeg> rec((size_t)m);
-    long long off = 0, fresh = 0, work = 0, slots = 0, tbl = 0;
+    long long off = 0, fresh = 0, work = 0, slots = 0, tbl = 0, copied_tokens = 0;
     for (int i = 0; i < m; ++i) {
         const long long T = p->len[segs[i]];
         ComposeSeg &r = rec[(size_t)i];
@@ -511,12 +515,13 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
             r.dst_tbl_start = (int)tbl;
             const long long items = nblk_of(p, T);
             work += items;
-            if (T % BS && i != m - 1) { fresh += 1; slots += 1; }
+            if (T % BS && i != m - 1) { fresh += 1; slots += 1; copied_tokens += T % BS; }
         } else {
             r.mode = 1;
             const long long items = (off + T - 1) / BS - off / BS + 1;
             work += items;
             slots += 2 * items;
+            copied_tokens += T;
             fresh += nblk_of(p, off + T) - nblk_of(p, off);
         }
         off += T;
@@ -542,7 +547,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     p->len[c] = off;
     p->live_ctx += 1;
     *out_ctx = c;
-    return run_copy(p, AAF_OP_COMPOSE, (int)slots, 0, 2 * p->g.L, st);
+    return run_copy(p, AAF_OP_COMPOSE, (int)slots, copied_tokens, st);
 }
 
 int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {
@@ -664,7 +669,7 @@ int aaf_kv_sync_status(aaf_kv_pool *p) {
 }
 
 int aaf_kv_set_copy_engine(aaf_kv_pool *p, int engine) {
-    if (!p || engine < AAF_ENGINE_AUTO || engine > AAF_ENGINE_BULK) return AAF_ERR_INVALID_ARG;
+    if (!p || engine < AAF_ENGINE_AUTO || engine > AAF_ENGINE_WARP) return AAF_ERR_INVALID_ARG;
     p->engine = engine;
     return AAF_OK;
 }

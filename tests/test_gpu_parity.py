@@ -15,7 +15,7 @@ from workloads.replay import replay
 
 pytestmark = pytest.mark.gpu
 
-VEC, BULK = 1, 2
+VEC, BULK, WARP = 1, 2, 3
 
 
 def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
@@ -39,7 +39,7 @@ def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
     return gpu, cpu
 
 
-@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("engine", [VEC, BULK, WARP])
 @pytest.mark.parametrize("unaligned", [False, True])
 def test_config1_tiny_pool(engine, unaligned):
     g, seed, ops = configs.config1(unaligned)
@@ -119,7 +119,7 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
     return outcomes
 
 
-@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("engine", [VEC, BULK, WARP])
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_random_operator_sequences_on_odd_geometry(engine, seed):
     outcomes = random_walk(ODD, 7000 + seed, 200, engine)
@@ -133,7 +133,7 @@ def test_random_operator_sequences_on_odd_geometry(engine, seed):
 MID = Geometry(4, 8, 128, 16, 2, 1024, 24, 256)
 
 
-@pytest.mark.parametrize("engine", [VEC, BULK])
+@pytest.mark.parametrize("engine", [VEC, BULK, WARP])
 @pytest.mark.parametrize("unaligned", [False, True])
 def test_fanout_with_8b_rows(engine, unaligned):
     T = 1019 if unaligned else 1024
