@@ -44,7 +44,7 @@ UNIT = "GB/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per algorithmic byte for the copy kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists)
-TRAFFIC_PER_ALGORITHMIC_BYTE = 0.91  # profiles/copy_vec_kernel_8b-small_ncu_full.md: (267.8 + 219.6) / (2 x 267.8) MB
+TRAFFIC_PER_ALGORITHMIC_BYTE = 0.90  # profiles/copy_bulk_kernel_8b-small_ncu_full.md: (267.9 + 216.4) / (2 x 267.8) MB
 
 
 def workload(name: str):
@@ -482,7 +482,7 @@ def main():
         dms = s1["copy_ms"][k] - s0["copy_ms"][k]
         per_class[k] = (2 * toks * g.bpt * args.steps / (dms * 1e-3) / 1e9) if dms > 0 else None
     roofline = {
-        "bound": "hbm", "kernel": "copy engine (aafkv::copy_vec_kernel / copy_bulk_kernel)", "achieved": achieved,
+        "bound": "hbm", "kernel": "copy engine (aafkv::copy_bulk_kernel; copy_warp_kernel for small pieces)", "achieved": achieved,
         "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
         "frac_of_nominal_8TBps": achieved / 8000.0,
         "traffic": (TRAFFIC_PER_ALGORITHMIC_BYTE * per_launch_bytes if TRAFFIC_PER_ALGORITHMIC_BYTE else None),
@@ -493,7 +493,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         layers = 2 if g.n_layers > 2 else g.n_layers
-        gbps, steps_c, dt, _ = oracle_rate(w, layers, budget_s=12.0, max_steps=50)
+        gbps, steps_c, dt, _ = oracle_rate(w, layers, budget_s=12.0, max_steps=2000)
         cpu_baseline = {"value": gbps, "unit": UNIT, "cores": 1, "kind": "oracle",
                         "sample": f"{layers} of {g.n_layers} layers of the same step, {steps_c} passes in {dt:.1f} s, "
                                   f"single thread of {len(os.sched_getaffinity(0))} available cores"}
