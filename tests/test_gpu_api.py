@@ -1,0 +1,129 @@
+"""C-ABI behaviour on a device: host-buffer entry points, descriptor compatibility, argument checks,
+statistics, engine selection.  Results are compared with the CPU oracle where bytes are involved."""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_10987_b200 import KVPool, binding
+from tests.helpers import GpuBackend, OracleBackend
+from workloads import configs, fill
+from workloads.configs import Geometry
+
+pytestmark = pytest.mark.gpu
+
+G = Geometry(3, 4, 64, 16, 2, 256, 8, 64)  # row 512 B, run 8 KiB
+SEED = 99
+
+
+def test_host_buffer_forms_match_the_oracle():
+    order = configs.free_order(SEED, G.n_blocks)
+    gpu = GpuBackend(G, SEED, free_order=order)
+    cpu = OracleBackend(G, SEED, free_order=order)
+    n = 333
+    payload = cpu.payload(SEED, 1, n)  # numpy uint8, full layers
+    h_src = torch.from_numpy(payload.copy()).pin_memory()
+    staging = torch.empty(n * G.bpt, dtype=torch.uint8, device=gpu.o.device)
+    st, c = gpu.o.import_host(h_src, n, staging)
+    assert st == 0
+    st2, c2 = cpu.imp(payload, n)
+    assert (st2, c2) == (0, c)
+    assert gpu.snapshot() == cpu.snapshot()
+    h_dst = torch.zeros(200 * G.bpt, dtype=torch.uint8).pin_memory()
+    assert gpu.o.materialize_host(c, 100, 300, h_dst, staging) == 0
+    torch.cuda.synchronize()
+    st, want = cpu.materialize(c, 100, 300)
+    assert np.array_equal(h_dst.numpy(), want)
+    assert np.array_equal(gpu.pool_layers(range(G.n_layers)), cpu.o.pool_view())
+    # too small host destination / staging
+    small = torch.zeros(16, dtype=torch.uint8).pin_memory()
+    assert gpu.o.materialize_host(c, 0, n, small, staging) == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.materialize_host(c, 0, n, h_src, staging[:1024]) == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.import_host(h_src, n, staging[:1024])[0] == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.snapshot() == cpu.snapshot()
+
+
+def test_incompatible_descriptor_is_refused_and_changes_nothing():
+    gpu = GpuBackend(G, SEED)
+    buf = gpu.payload(SEED, 1, 40)
+    before = gpu.snapshot()
+    for field, value in (("model_id", 7), ("config_hash", 7), ("n_layers", 2), ("head_dim", 32), ("elt_bytes", 4)):
+        d = gpu.o.xfer_desc(40)
+        setattr(d, field, value)
+        assert gpu.o.imp(buf, 40, desc=d)[0] == binding.AAF_ERR_INCOMPAT, field
+    d = gpu.o.xfer_desc(0)
+    assert gpu.o.imp(buf, 0, desc=d)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.snapshot() == before
+    # the descriptor materialize fills in is accepted back by import (transfer round trip, positions carried)
+    st, c = gpu.o.imp(buf, 40)
+    out = torch.empty(30 * G.bpt, dtype=torch.uint8, device=gpu.o.device)
+    xd = binding.aaf_kv_xfer_desc()
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert binding.aaf_kv_materialize(gpu.o.h, c, 5, 35, out.data_ptr(), out.numel(), C.byref(xd), stream) == 0
+    assert (xd.pos_start, xd.n_tokens, xd.n_layers) == (5, 30, G.n_layers)
+    assert gpu.o.imp(out, 30, desc=xd)[0] == 0
+
+
+def test_pointer_and_range_checks():
+    gpu = GpuBackend(G, SEED)
+    buf = gpu.payload(SEED, 1, 40)
+    st, c = gpu.o.imp(buf, 40)
+    out = torch.empty(40 * G.bpt + 64, dtype=torch.uint8, device=gpu.o.device)
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    mis = out.data_ptr() + 8
+    assert binding.aaf_kv_materialize(gpu.o.h, c, 0, 40, mis, 40 * G.bpt, None, stream) == binding.AAF_ERR_INVALID_ARG
+    assert binding.aaf_kv_materialize(gpu.o.h, c, 0, 40, out.data_ptr(), 40 * G.bpt - 1, None, stream) == \
+        binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.materialize(c, 0, 41)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.materialize(c, 7, 7)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.materialize(5, 0, 1)[0] == binding.AAF_ERR_BAD_CTX
+    d = gpu.o.xfer_desc(40)
+    out_ctx = C.c_int32(-1)
+    assert binding.aaf_kv_import(gpu.o.h, buf.data_ptr() + 4, C.byref(d), C.byref(out_ctx), stream) == \
+        binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.set_copy_engine(9) == binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.fork(c, 0)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.fork(c, 5000)[0] == binding.AAF_ERR_TOO_MANY
+    assert gpu.o.sync_status() == 0
+
+
+def test_out_of_blocks_is_exact_after_evictions_the_host_did_not_count():
+    """The host only keeps a lower bound of the free count (evict does not raise it); a request the
+    bound cannot prove must be decided against the device's real count, not refused."""
+    g = Geometry(1, 1, 8, 4, 2, 16, 8, 16)
+    gpu = GpuBackend(g, SEED)
+    cpu = OracleBackend(g, SEED)
+    mk = lambda be, s, n: be.payload(SEED, s, n)
+    for be in (gpu, cpu):
+        assert be.imp(mk(be, 1, 40), 40) == (0, 0)       # 10 blocks
+        assert be.imp(mk(be, 2, 18), 18) == (0, 1)       # 5 blocks (tail half full) -> 1 free
+        assert be.imp(mk(be, 3, 8), 8)[0] == binding.AAF_ERR_OOM_BLOCKS
+        assert be.evict([0])[0] == 0                     # 11 free, the host's bound still says 1
+        assert be.imp(mk(be, 4, 44), 44) == (0, 0)       # exactly 11 blocks: must succeed
+        assert be.imp(mk(be, 5, 1), 1)[0] == binding.AAF_ERR_OOM_BLOCKS
+        # append whose worst case (COW + 1) does not fit but whose real need (in place, 0 new blocks) does
+        assert be.fork(1, 1) == (0, [2])
+        assert be.evict([2])[0] == 0                     # tail of ctx 1 is unshared again
+        assert be.append([1], [2], [mk(be, 6, 2)])[0] == 0  # 18 -> 20 tokens in place: the real need is 0 blocks
+        assert be.append([1], [1], [mk(be, 7, 1)])[0] == binding.AAF_ERR_OOM_BLOCKS  # would need a 6th block
+    assert gpu.snapshot() == cpu.snapshot()
+    assert np.array_equal(gpu.pool_layers([0]), cpu.o.pool_view())
+
+
+def test_stats_and_launch_counters():
+    gpu = GpuBackend(G, SEED)
+    gpu.o.set_timing(True)
+    st, c = gpu.o.imp(gpu.payload(SEED, 1, 100), 100)
+    gpu.o.materialize(c, 0, 100)
+    kids = gpu.o.fork(c, 2)[1]
+    gpu.o.append([kids[0]], [5], [gpu.payload(SEED, 2, 5)])
+    s = gpu.o.stats()
+    assert s["copy_launches"] == {"materialize": 1, "import": 1, "append": 1, "compose": 0}
+    assert s["timed_launches"] == s["copy_launches"]
+    assert all(v > 0 for k, v in s["copy_ms"].items() if k != "compose")
+    assert s["meta_launches"] == 4 and s["cow_count"] == 1 and s["live_ctx"] == 3
+    assert s["payload_bytes"] == (100 + 100 + 5 + 100 % 16) * G.bpt
+    assert s["live_blocks"] == 7 + 1 and s["free_blocks"] == G.n_blocks - 8
