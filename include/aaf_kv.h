@@ -244,6 +244,14 @@ int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t layer_stride_by
                                int32_t n_blocks, const int32_t *block_table_host, int32_t n_table_blocks,
                                int64_t tok_begin, int64_t tok_end, void *dst_dev, size_t dst_bytes, void *stream);
 
+/* Test hook for the failure path of the device-side waits (no paper counterpart).  Every wait in the
+ * library's kernels is bounded: when its limit expires the kernel records AAF_ERR_TIMEOUT in the
+ * sticky status word and returns, so the context stays usable.  This call launches a one-thread
+ * kernel that waits, for at most limit_cycles SM clock cycles (1 .. 2^31), on a barrier nothing ever
+ * signals, so that a test can watch the limit expire: aaf_kv_sync_status then returns
+ * AAF_ERR_TIMEOUT once, and the pool keeps working.  Nothing faults, traps or hangs. */
+int aaf_kv_debug_expire_wait(aaf_kv_pool *pool, uint64_t limit_cycles, void *stream);
+
 const char *aaf_kv_strerror(int status);
 
 #ifdef __cplusplus

@@ -81,6 +81,7 @@ SYMBOLS = {
     "aaf_kv_set_timing": (C.c_int, [_vp, C.c_int]),
     "aaf_kv_materialize_noalloc": (C.c_int, [_vp, _sz, _i32, _i32, _i32, _i32, _i32, _i32, _p32, _i32, _i64, _i64, _vp,
                                              _sz, _vp]),
+    "aaf_kv_debug_expire_wait": (C.c_int, [_vp, C.c_uint64, _vp]),
     "aaf_kv_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -138,6 +139,7 @@ def aaf_kv_materialize_noalloc(pool_base, layer_stride, n_layers, n_kv_heads, he
     return _fn("aaf_kv_materialize_noalloc")(pool_base, layer_stride, n_layers, n_kv_heads, head_dim, block_size,
                                              elt_bytes, n_blocks, block_table_host, n_table_blocks, t0, t1, dst,
                                              dst_bytes, stream)
+def aaf_kv_debug_expire_wait(pool, limit_cycles, stream): return _fn("aaf_kv_debug_expire_wait")(pool, limit_cycles, stream)
 def aaf_kv_strerror(status): return _fn("aaf_kv_strerror")(status).decode()
 
 

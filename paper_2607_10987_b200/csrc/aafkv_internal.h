@@ -100,6 +100,7 @@ struct CopyTuning {
     long long auto_bulk_min_piece; // AUTO: mean piece size from which the bulk engine is used
 };
 cudaError_t copy_tuning_init(long long run, CopyTuning *t);
+cudaError_t launch_expire_wait(const DevState &s, long long limit_cycles, cudaStream_t st);
 cudaError_t launch_copy(int engine, const CopyTuning &t, const Geom &g, const DevState &s, int n_slots, int plane0,
                         int n_planes, long long avg_piece_bytes, int sm_count, cudaStream_t st);
 

@@ -152,14 +152,30 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
         : "memory");
     return ok != 0;
 }
-// bounded wait: false if the phase did not complete within BULK_WAIT_CYCLES
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
+// bounded wait: false if the phase did not complete within `limit` SM clock cycles
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, long long limit = BULK_WAIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > BULK_WAIT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
+}
+
+// Test hook: exercises the give-up path of the bounded wait without any fault.  One thread waits, with a
+// short limit, on an mbarrier that nothing ever arrives at; when the limit expires it records
+// AAF_ERR_TIMEOUT in the status word and returns, exactly as the bulk engine would.
+__global__ void expire_wait_kernel(DevCtl *ctl, long long limit_cycles) {
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x != 0) return;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_bounded(smem_u32(&bar), 0, limit_cycles)) atomicCAS(&ctl->status, 0, (int)AAF_ERR_TIMEOUT);
+}
+
+cudaError_t launch_expire_wait(const DevState &s, long long limit_cycles, cudaStream_t st) {
+    expire_wait_kernel<<<1, 32, 0, st>>>(s.ctl, limit_cycles);
+    return cudaGetLastError();
 }
 // L2 policy for data that is touched once: mark the lines evict-first so that the stream does not push
 // other tenants' data out of the 126 MB L2

@@ -674,6 +674,15 @@ int aaf_kv_set_copy_engine(aaf_kv_pool *p, int engine) {
     return AAF_OK;
 }
 
+int aaf_kv_debug_expire_wait(aaf_kv_pool *p, uint64_t limit_cycles, void *stream) {
+    if (!p || limit_cycles == 0 || limit_cycles > (1ull << 31)) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    p->meta_launches += 1;
+    return launch_expire_wait(p->s, (long long)limit_cycles, st) == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
+}
+
 int aaf_kv_set_timing(aaf_kv_pool *p, int enable) {
     if (!p) return AAF_ERR_INVALID_ARG;
     p->timing = enable != 0;

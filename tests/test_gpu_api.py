@@ -127,3 +127,25 @@ def test_stats_and_launch_counters():
     assert s["meta_launches"] == 4 and s["cow_count"] == 1 and s["live_ctx"] == 3
     assert s["payload_bytes"] == (100 + 100 + 5 + 100 % 16) * G.bpt
     assert s["live_blocks"] == 7 + 1 and s["free_blocks"] == G.n_blocks - 8
+
+
+def test_bounded_wait_expires_with_a_status_and_the_pool_keeps_working():
+    """Failure detection without a fault: a device-side wait that nothing will ever satisfy gives up after
+    its limit, records AAF_ERR_TIMEOUT, and the next operators run normally."""
+    gpu = GpuBackend(G, SEED)
+    cpu = OracleBackend(G, SEED)
+    pay = lambda be: be.payload(SEED, 1, 50)
+    assert gpu.imp(pay(gpu), 50) == cpu.imp(pay(cpu), 50) == (0, 0)
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert binding.aaf_kv_debug_expire_wait(gpu.o.h, 2_000_000, stream) == 0  # about a millisecond
+    assert gpu.o.sync_status() == binding.AAF_ERR_TIMEOUT
+    assert gpu.o.sync_status() == 0, "the status is sticky until read, then cleared"
+    assert binding.aaf_kv_debug_expire_wait(gpu.o.h, 0, stream) == binding.AAF_ERR_INVALID_ARG
+    for be in (gpu, cpu):
+        assert be.fork(0, 2)[0] == 0
+        assert be.append([1], [7], [be.payload(SEED, 2, 7)])[0] == 0
+    st, got = gpu.materialize(1, 0, 57)
+    st2, want = cpu.materialize(1, 0, 57)
+    assert st == st2 == 0
+    assert np.array_equal(gpu.buf_layers(got, 57, range(G.n_layers)).reshape(-1), want)
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
