@@ -291,6 +291,53 @@ def extra_report(args):
             out["copy_all" if copy_all else "share"] = rep
             del be
             torch.cuda.empty_cache()
+    elif args.workload == "transfer":
+        # pack / unpack against host memory: one shot versus chunked with per-chunk completion flags
+        g, seed, T = configs.LLAMA8B, configs.SEED_BASE + 2, 8187
+        g = configs.Geometry(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, 4096, 8, 1024)
+        be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False)
+        pool = be.o
+        h_src = torch.empty(T * g.bpt, dtype=torch.uint8).pin_memory()
+        h_src.copy_(be.payload(seed, 1, T))
+        h_dst = torch.empty(T * g.bpt, dtype=torch.uint8).pin_memory()
+        staging = torch.empty(T * g.bpt, dtype=torch.uint8, device=dev)
+        flags = torch.zeros(1024, dtype=torch.int32).pin_memory()
+        fl = flags.numpy()
+        st, c = pool.import_host(h_src, T, staging)
+        assert st == 0
+        rep = {}
+        for chunk in (0, 512, 1024, 2048):
+            first, total, imp = [], [], []
+            for it in range(args.warmup + args.steps):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                if chunk:
+                    st, nch = pool.materialize_host_chunked(c, 0, T, h_dst, staging, chunk, flags)
+                    assert st == 0
+                    while fl[0] == 0:
+                        pass
+                    t_first = time.perf_counter() - t0
+                else:
+                    assert pool.materialize_host(c, 0, T, h_dst, staging) == 0
+                    t_first = None
+                torch.cuda.synchronize()
+                t_total = time.perf_counter() - t0
+                t1 = time.perf_counter()
+                st, c2 = pool.import_host_chunked(h_dst, T, staging, chunk) if chunk else pool.import_host(h_dst, T, staging)
+                assert st == 0
+                torch.cuda.synchronize()
+                t_imp = time.perf_counter() - t1
+                pool.evict([c2])
+                if it >= args.warmup:
+                    total.append(t_total); imp.append(t_imp)
+                    if t_first is not None:
+                        first.append(t_first)
+            rep["one_shot" if not chunk else f"chunk_{chunk}_tokens"] = {
+                "materialize_to_host_ms": 1e3 * sum(total) / len(total),
+                "first_chunk_on_host_ms": (1e3 * sum(first) / len(first)) if first else None,
+                "import_from_host_ms": 1e3 * sum(imp) / len(imp)}
+        assert torch.equal(h_dst, h_src)
+        out.update({"context_tokens": T, "bytes_each_way_GB": T * g.bpt / 1e9, "modes": rep})
     else:  # churn
         bs, cap, seed = args.block_size, 32768, configs.SEED_BASE + 5
         small = lambda nb: configs.Geometry(1, 1, 8, bs, 2, nb, 80, cap // bs)
@@ -332,13 +379,13 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer"])
     ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST per CTA, 2 cp.async.bulk, 3 vector LD/ST per warp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    if args.workload in ("cow", "compose", "churn"):
+    if args.workload in ("cow", "compose", "churn", "transfer"):
         return extra_report(args)
     w = workload(args.workload)
     if args.impl == "reference":

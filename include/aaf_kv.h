@@ -204,6 +204,29 @@ int aaf_kv_materialize_host(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin,
 int aaf_kv_import_host(aaf_kv_pool *pool, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
                        size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream);
 
+/* Chunked, overlapped forms of the host transfer (Sec. 5.4: the transport overlaps communication
+ * with computation, and consumers may start as blocks arrive).  The token range is cut into chunks
+ * of chunk_tokens tokens (a multiple of block_size, counted from the block that holds tok_begin);
+ * while one chunk crosses PCIe on a library-owned copy stream, the kernel for the next chunk runs on
+ * `stream`.  Results are byte-identical to the unchunked forms.
+ *   materialize: done_flags_host (host, pinned recommended, may be NULL; flags_cap entries) receives
+ *   one completion flag per chunk: the library zeroes the flags, and flag c becomes 1, in stream
+ *   order, after chunk c's bytes have landed in dst_host, so a consumer (a network sender) can poll
+ *   and forward chunk c while later chunks are still being packed.  Chunk c covers the columns of
+ *   blocks [c * chunk_tokens / BS, ...) of the range in every (layer, K/V) plane of dst_host.
+ *   *n_chunks_out (host, may be NULL) receives the number of chunks.  `stream` is complete only
+ *   when the last chunk has landed.
+ *   import: blocks are allocated up front; chunk c is scattered as soon as it has arrived.
+ * Errors as for the unchunked forms, plus INVALID_ARG for a chunk_tokens that is not a positive
+ * multiple of block_size and DST_TOO_SMALL for too few flags. */
+int aaf_kv_materialize_host_chunked(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end,
+                                    void *dst_host, size_t dst_bytes, void *staging_dev, size_t staging_bytes,
+                                    int32_t chunk_tokens, uint32_t *done_flags_host, int32_t flags_cap,
+                                    int32_t *n_chunks_out, aaf_kv_xfer_desc *out_desc, void *stream);
+int aaf_kv_import_host_chunked(aaf_kv_pool *pool, const void *src_host, const aaf_kv_xfer_desc *desc,
+                               void *staging_dev, size_t staging_bytes, int32_t chunk_tokens, aaf_ctx_t *out_ctx,
+                               void *stream);
+
 /* Introspection (metadata catalog of App. A.2).  These synchronise the pool's stream. */
 int aaf_kv_ctx_len(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t *n_tokens);
 int aaf_kv_get_table(aaf_kv_pool *pool, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks);

@@ -71,6 +71,9 @@ SYMBOLS = {
     "aaf_kv_evict": (C.c_int, [_vp, _i32, _p32, _vp]),
     "aaf_kv_materialize_host": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _p32, _vp]),
+    "aaf_kv_materialize_host_chunked": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, _i32, C.POINTER(C.c_uint32),
+                                                  _i32, _p32, C.POINTER(aaf_kv_xfer_desc), _vp]),
+    "aaf_kv_import_host_chunked": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _i32, _p32, _vp]),
     "aaf_kv_ctx_len": (C.c_int, [_vp, _i32, C.POINTER(_i64)]),
     "aaf_kv_get_table": (C.c_int, [_vp, _i32, _p32, _i32, _p32]),
     "aaf_kv_get_refcounts": (C.c_int, [_vp, _p32]),
@@ -124,6 +127,12 @@ def aaf_kv_materialize_host(pool, ctx, t0, t1, dst_host, dst_bytes, staging, sta
     return _fn("aaf_kv_materialize_host")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream)
 def aaf_kv_import_host(pool, src_host, desc, staging, staging_bytes, out_ctx, stream):
     return _fn("aaf_kv_import_host")(pool, src_host, desc, staging, staging_bytes, out_ctx, stream)
+def aaf_kv_materialize_host_chunked(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, chunk_tokens,
+                                    done_flags, flags_cap, n_chunks_out, out_desc, stream):
+    return _fn("aaf_kv_materialize_host_chunked")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes,
+                                                  chunk_tokens, done_flags, flags_cap, n_chunks_out, out_desc, stream)
+def aaf_kv_import_host_chunked(pool, src_host, desc, staging, staging_bytes, chunk_tokens, out_ctx, stream):
+    return _fn("aaf_kv_import_host_chunked")(pool, src_host, desc, staging, staging_bytes, chunk_tokens, out_ctx, stream)
 def aaf_kv_ctx_len(pool, ctx, out): return _fn("aaf_kv_ctx_len")(pool, ctx, out)
 def aaf_kv_get_table(pool, ctx, out, cap, n_blocks): return _fn("aaf_kv_get_table")(pool, ctx, out, cap, n_blocks)
 def aaf_kv_get_refcounts(pool, out): return _fn("aaf_kv_get_refcounts")(pool, out)
@@ -268,6 +277,25 @@ class KVPool:
         out = C.c_int32(-1)
         st = aaf_kv_import_host(self.h, src_host.data_ptr(), C.byref(xd), staging.data_ptr(),
                                 staging.numel() * staging.element_size(), C.byref(out), self._stream())
+        return st, (out.value if st == AAF_OK else None)
+
+    def materialize_host_chunked(self, ctx, t0, t1, dst_host, staging, chunk_tokens, flags=None):
+        """flags: pinned torch int32 tensor receiving one completion flag per chunk (or None)."""
+        nch = C.c_int32(0)
+        fptr = C.cast(flags.data_ptr(), C.POINTER(C.c_uint32)) if flags is not None else None
+        st = aaf_kv_materialize_host_chunked(self.h, ctx, t0, t1, dst_host.data_ptr(),
+                                             dst_host.numel() * dst_host.element_size(), staging.data_ptr(),
+                                             staging.numel() * staging.element_size(), chunk_tokens, fptr,
+                                             flags.numel() if flags is not None else 0, C.byref(nch), None,
+                                             self._stream())
+        return st, nch.value
+
+    def import_host_chunked(self, src_host, n, staging, chunk_tokens):
+        xd = self.xfer_desc(n)
+        out = C.c_int32(-1)
+        st = aaf_kv_import_host_chunked(self.h, src_host.data_ptr(), C.byref(xd), staging.data_ptr(),
+                                        staging.numel() * staging.element_size(), chunk_tokens, C.byref(out),
+                                        self._stream())
         return st, (out.value if st == AAF_OK else None)
 
     # ------------------------------------------------------------------ introspection

@@ -31,7 +31,9 @@ struct DevCtl {
     unsigned long long cow_count;
     long long peak_live;
     unsigned long long probe_need;     // dry-run result of the append planner
-    unsigned long long pad[9];
+    unsigned int one;                  // constant 1: source of the host-visible chunk completion flags
+    unsigned int pad32;
+    unsigned long long pad[8];
 };
 static_assert(sizeof(DevCtl) == 128, "DevCtl layout");
 

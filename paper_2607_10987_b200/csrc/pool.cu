@@ -103,6 +103,10 @@ struct aaf_kv_pool {
     long long timed_launches[AAF_OP_CLASSES] = {};
     std::vector<TimedLaunch> pending;
     std::vector<cudaEvent_t> spare_events;
+    // chunked host transfers: a second stream for the PCIe copies and ordering events
+    cudaStream_t xfer_stream = nullptr;
+    std::vector<cudaEvent_t> order_events;  // created on demand, reused round-robin
+    size_t next_order_event = 0;
 };
 
 namespace {
@@ -176,8 +180,10 @@ void drain_timing(aaf_kv_pool *p) {
 }
 
 // copy-engine launch for one operator class over planes [plane0, plane0 + n_planes)
-int run_copy(aaf_kv_pool *p, int cls, int n_slots, long long payload_tokens, cudaStream_t st) {
+int run_copy(aaf_kv_pool *p, int cls, int n_slots, long long payload_tokens, cudaStream_t st, int piece0 = 0) {
     const int plane0 = 0, n_planes = 2 * p->g.L;
+    DevState view = p->s;
+    view.pieces += piece0;  // a launch may cover a sub-range of the planned pieces (chunked transfers)
     const long long avg_piece = n_slots > 0 ? payload_tokens * p->g.row / n_slots : 0;
     if (n_slots <= 0) return AAF_OK;
     TimedLaunch t{};
@@ -187,7 +193,7 @@ int run_copy(aaf_kv_pool *p, int cls, int n_slots, long long payload_tokens, cud
         t.cls = cls;
         cudaEventRecord(t.start, st);
     }
-    const cudaError_t e = launch_copy(p->engine, p->tuning, p->g, p->s, n_slots, plane0, n_planes, avg_piece, p->sm_count, st);
+    const cudaError_t e = launch_copy(p->engine, p->tuning, p->g, view, n_slots, plane0, n_planes, avg_piece, p->sm_count, st);
     if (p->timing) {
         cudaEventRecord(t.stop, st);
         p->pending.push_back(t);
@@ -253,6 +259,31 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
     p->live_ctx += 1;
     *out_ctx = c;
     return run_copy(p, AAF_OP_IMPORT, (int)nb, n, st);
+}
+
+cudaEvent_t order_event(aaf_kv_pool *p) {
+    if (p->order_events.size() < 64) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        p->order_events.push_back(e);
+        return e;
+    }
+    cudaEvent_t e = p->order_events[p->next_order_event];
+    p->next_order_event = (p->next_order_event + 1) % p->order_events.size();
+    return e;
+}
+
+bool ensure_xfer_stream(aaf_kv_pool *p) {
+    if (p->xfer_stream) return true;
+    return cudaStreamCreateWithFlags(&p->xfer_stream, cudaStreamNonBlocking) == cudaSuccess;
+}
+
+// column slab [col0, col0 + cnt) tokens of an n-token transfer buffer: 2L rows of cnt*row bytes, pitch n*row
+cudaError_t copy_slab(aaf_kv_pool *p, char *dst, const char *src, long long n, long long col0, long long cnt,
+                      cudaMemcpyKind kind, cudaStream_t st) {
+    const size_t pitch = (size_t)(n * p->g.row);
+    return cudaMemcpy2DAsync(dst + col0 * p->g.row, pitch, src + col0 * p->g.row, pitch, (size_t)(cnt * p->g.row),
+                             (size_t)(2 * p->g.L), kind, st);
 }
 
 }  // namespace
@@ -326,6 +357,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     DevCtl ctl;
     memset(&ctl, 0, sizeof(ctl));
     ctl.tail = (unsigned long long)desc->n_blocks;
+    ctl.one = 1u;
     ok = ok && cudaMemset(ws, 0, lay.tables) == cudaSuccess;
     ok = ok && cudaMemcpy(p->s.ctl, &ctl, sizeof(ctl), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(p->s.ring, ring.data(), sizeof(int) * ring.size(), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -349,6 +381,11 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
         cudaEventDestroy(t.stop);
     }
     for (auto e : p->spare_events) cudaEventDestroy(e);
+    if (p->xfer_stream) {
+        cudaStreamSynchronize(p->xfer_stream);
+        cudaStreamDestroy(p->xfer_stream);
+    }
+    for (auto e : p->order_events) cudaEventDestroy(e);
     for (int i = 0; i < ARG_SLOTS; ++i)
         if (p->slot_ev[i]) cudaEventDestroy(p->slot_ev[i]);
     if (p->args) cudaFreeHost(p->args);
@@ -394,6 +431,101 @@ int aaf_kv_import_host(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_d
     if (desc->n_tokens >= 1 && (unsigned long long)staging_bytes < (unsigned long long)(desc->n_tokens * bpt_of(p)))
         return AAF_ERR_DST_TOO_SMALL;
     return import_impl(p, staging_dev, desc, out_ctx, static_cast<cudaStream_t>(stream), src_host);
+}
+
+int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void *dst_host,
+                                    size_t dst_bytes, void *staging_dev, size_t staging_bytes, int32_t chunk_tokens,
+                                    uint32_t *done_flags_host, int32_t flags_cap, int32_t *n_chunks_out,
+                                    aaf_kv_xfer_desc *out_desc, void *stream) {
+    if (!p || !dst_host || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0) return AAF_ERR_INVALID_ARG;
+    if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
+    if (!aligned16(staging_dev) || t0 < 0 || t0 >= t1 || t1 > p->len[ctx]) return AAF_ERR_INVALID_ARG;
+    const long long n = t1 - t0;
+    if ((unsigned long long)dst_bytes < (unsigned long long)(n * bpt_of(p)) ||
+        (unsigned long long)staging_bytes < (unsigned long long)(n * bpt_of(p)))
+        return AAF_ERR_DST_TOO_SMALL;
+    const int BS = p->g.BS;
+    const long long j0 = t0 / BS, j1 = (t1 - 1) / BS;
+    const int n_slots = (int)(j1 - j0 + 1), per_chunk = chunk_tokens / BS;
+    const int n_chunks = (n_slots + per_chunk - 1) / per_chunk;
+    if (done_flags_host && flags_cap < n_chunks) return AAF_ERR_DST_TOO_SMALL;
+    DeviceGuard guard(p->device);
+    if (!ensure_xfer_stream(p)) return AAF_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    if (done_flags_host)
+        for (int c = 0; c < n_chunks; ++c) done_flags_host[c] = 0;
+    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(staging_dev), st) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    bool ok = true;
+    for (int c = 0; c < n_chunks && ok; ++c) {
+        const int s0 = c * per_chunk, s1 = std::min(n_slots, s0 + per_chunk);
+        const long long lo = std::max<long long>(t0, (j0 + s0) * BS), hi = std::min<long long>(t1, (j0 + s1) * BS);
+        ok = run_copy(p, AAF_OP_MATERIALIZE, s1 - s0, hi - lo, st, s0) == AAF_OK;  // gather of this chunk's blocks
+        cudaEvent_t ev = order_event(p);
+        ok = ok && ev && cudaEventRecord(ev, st) == cudaSuccess &&
+             cudaStreamWaitEvent(p->xfer_stream, ev, 0) == cudaSuccess;
+        // while the next chunk is gathered, this one crosses PCIe
+        ok = ok && copy_slab(p, static_cast<char *>(dst_host), static_cast<const char *>(staging_dev), n, lo - t0,
+                             hi - lo, cudaMemcpyDeviceToHost, p->xfer_stream) == cudaSuccess;
+        if (ok && done_flags_host)  // completion flag of the chunk, written in stream order after its bytes
+            ok = cudaMemcpyAsync(&done_flags_host[c], &p->s.ctl->one, sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                                 p->xfer_stream) == cudaSuccess;
+    }
+    // the caller's stream is complete only when the last chunk has landed
+    cudaEvent_t fin = order_event(p);
+    ok = ok && fin && cudaEventRecord(fin, p->xfer_stream) == cudaSuccess && cudaStreamWaitEvent(st, fin, 0) == cudaSuccess;
+    if (!ok) return AAF_ERR_CUDA;
+    if (n_chunks_out) *n_chunks_out = n_chunks;
+    if (out_desc) fill_desc(p, out_desc, t0, n);
+    return AAF_OK;
+}
+
+int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
+                               size_t staging_bytes, int32_t chunk_tokens, aaf_ctx_t *out_ctx, void *stream) {
+    if (!p || !src_host || !desc || !out_ctx || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0 ||
+        !aligned16(staging_dev))
+        return AAF_ERR_INVALID_ARG;
+    if (!compatible(p, desc)) return AAF_ERR_INCOMPAT;
+    const long long n = desc->n_tokens;
+    if (n < 1) return AAF_ERR_INVALID_ARG;
+    if ((unsigned long long)staging_bytes < (unsigned long long)(n * bpt_of(p))) return AAF_ERR_DST_TOO_SMALL;
+    const long long nb = nblk_of(p, n);
+    if (nb > p->g.max_blk) return AAF_ERR_TOO_LONG;
+    const int c = smallest_free_ctx(p);
+    if (c < 0) return AAF_ERR_OOM_CTX;
+    DeviceGuard guard(p->device);
+    if (!ensure_xfer_stream(p)) return AAF_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int rc0 = ensure_free(p, nb, st);
+    if (rc0 != AAF_OK) return rc0;
+    p->last_stream = st;
+    // the PCIe stream may only overwrite the staging buffer after everything already queued on the
+    // caller's stream (earlier readers of that buffer) has run
+    cudaEvent_t start = order_event(p);
+    bool ok = start && cudaEventRecord(start, st) == cudaSuccess &&
+              cudaStreamWaitEvent(p->xfer_stream, start, 0) == cudaSuccess;
+    ok = ok && launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(staging_dev), st) == cudaSuccess;
+    if (!ok) return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    p->free_lb -= nb;
+    p->len[c] = n;
+    p->live_ctx += 1;
+    *out_ctx = c;
+    const int BS = p->g.BS, per_chunk = chunk_tokens / BS;
+    for (long long s0 = 0; s0 < nb && ok; s0 += per_chunk) {
+        const long long s1 = std::min<long long>(nb, s0 + per_chunk);
+        const long long lo = s0 * BS, hi = std::min<long long>(n, s1 * BS);
+        ok = copy_slab(p, static_cast<char *>(staging_dev), static_cast<const char *>(src_host), n, lo, hi - lo,
+                       cudaMemcpyHostToDevice, p->xfer_stream) == cudaSuccess;
+        cudaEvent_t ev = order_event(p);
+        ok = ok && ev && cudaEventRecord(ev, p->xfer_stream) == cudaSuccess &&
+             cudaStreamWaitEvent(st, ev, 0) == cudaSuccess;
+        // scatter of the chunk that has arrived, while the next one crosses PCIe
+        ok = ok && run_copy(p, AAF_OP_IMPORT, (int)(s1 - s0), hi - lo, st, (int)s0) == AAF_OK;
+    }
+    return ok ? AAF_OK : AAF_ERR_CUDA;
 }
 
 int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream) {

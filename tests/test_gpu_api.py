@@ -149,3 +149,35 @@ def test_bounded_wait_expires_with_a_status_and_the_pool_keeps_working():
     assert st == st2 == 0
     assert np.array_equal(gpu.buf_layers(got, 57, range(G.n_layers)).reshape(-1), want)
     assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+
+
+@pytest.mark.parametrize("chunk_tokens", [16, 32, 160, 4096])
+def test_chunked_host_transfer_is_byte_identical_and_flags_every_chunk(chunk_tokens):
+    order = configs.free_order(SEED, G.n_blocks)
+    gpu = GpuBackend(G, SEED, free_order=order)
+    cpu = OracleBackend(G, SEED, free_order=order)
+    n = 333
+    payload = cpu.payload(SEED, 1, n)
+    h_src = torch.from_numpy(payload.copy()).pin_memory()
+    staging = torch.empty(n * G.bpt, dtype=torch.uint8, device=gpu.o.device)
+    # chunked import: H2D of chunk c+1 overlaps the scatter of chunk c
+    st, c = gpu.o.import_host_chunked(h_src, n, staging, chunk_tokens)
+    assert (st, c) == (0, 0) and cpu.imp(payload, n) == (0, 0)
+    assert gpu.snapshot() == cpu.snapshot()
+    assert np.array_equal(gpu.pool_layers(range(G.n_layers)), cpu.o.pool_view())
+    # chunked materialize of an unaligned range, one completion flag per chunk
+    t0, t1 = 37, 300
+    h_dst = torch.zeros((t1 - t0) * G.bpt, dtype=torch.uint8).pin_memory()
+    flags = torch.full((64,), 7, dtype=torch.int32).pin_memory()
+    st, n_chunks = gpu.o.materialize_host_chunked(c, t0, t1, h_dst, staging, chunk_tokens, flags)
+    assert st == 0
+    blocks = (t1 - 1) // 16 - t0 // 16 + 1
+    assert n_chunks == -(-blocks // (chunk_tokens // 16))
+    torch.cuda.synchronize()
+    assert flags[:n_chunks].tolist() == [1] * n_chunks and flags[n_chunks:].tolist() == [7] * (64 - n_chunks)
+    assert np.array_equal(h_dst.numpy(), cpu.materialize(c, t0, t1)[1])
+    # argument checks
+    assert gpu.o.materialize_host_chunked(c, t0, t1, h_dst, staging, 24, flags)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.o.materialize_host_chunked(c, t0, t1, h_dst, staging, 16, flags[:3])[0] == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.import_host_chunked(h_src, n, staging, 0)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
