@@ -55,6 +55,9 @@ typedef struct kvo_pool {
     uint64_t head, tail;  /* free count = tail - head                 */
     int32_t *table;       /* [max_ctx][max_blk]                       */
     int64_t *len;         /* [max_ctx] tokens; -1 = slot is free      */
+    int64_t *reuse;       /* [max_ctx] times the state was read by fork / materialize / compose   */
+    int64_t *last_access; /* [max_ctx] logical clock of the last operator that used the state     */
+    int64_t clock;        /* logical clock: number of successful state-touching operators so far  */
     int64_t peak_live;    /* max over time of NB - free (Mem_KV in blocks, Sec. 6.2) */
     int64_t cow_count;    /* copy-on-write events so far              */
     int64_t rows_copied;  /* rows moved by memcpy so far              */
@@ -126,6 +129,12 @@ static int has_duplicates(const int32_t *v, int32_t n) {
     return 0;
 }
 
+/* Catalog bookkeeping (metadata catalog of App. A.2: "last_access: timestamp or logical clock for
+ * eviction"; the reuse term of the eviction score).  The logical clock counts successful
+ * state-touching operators; an operator stamps every state it reads, writes or creates. */
+static void born(kvo_pool *p, int32_t c) { p->reuse[c] = 0; p->last_access[c] = p->clock; }
+static void read_by_other(kvo_pool *p, int32_t c) { p->reuse[c] += 1; p->last_access[c] = p->clock; }
+
 /* ---------------------------------------------------------------- create / destroy */
 
 /* Pool creation: no block referenced, free ring = free_order (a permutation of
@@ -144,7 +153,9 @@ kvo_pool *kvo_create(int32_t L, int32_t H, int32_t D, int32_t BS, int32_t E, int
     p->ring = (int32_t *)malloc((size_t)NB * sizeof(int32_t));
     p->table = (int32_t *)calloc((size_t)max_ctx * max_blk, sizeof(int32_t));
     p->len = (int64_t *)malloc((size_t)max_ctx * sizeof(int64_t));
-    if (!p->pool || !p->refcount || !p->ring || !p->table || !p->len) return NULL;
+    p->reuse = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
+    p->last_access = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
+    if (!p->pool || !p->refcount || !p->ring || !p->table || !p->len || !p->reuse || !p->last_access) return NULL;
     for (int32_t i = 0; i < NB; ++i) p->ring[i] = free_order ? free_order[i] : i;
     for (int32_t c = 0; c < max_ctx; ++c) p->len[c] = -1;
     p->head = 0;
@@ -155,6 +166,7 @@ kvo_pool *kvo_create(int32_t L, int32_t H, int32_t D, int32_t BS, int32_t E, int
 void kvo_destroy(kvo_pool *p) {
     if (!p) return;
     free(p->pool); free(p->refcount); free(p->ring); free(p->table); free(p->len);
+    free(p->reuse); free(p->last_access);
     free(p);
 }
 
@@ -167,6 +179,9 @@ kvo_pool *kvo_clone(const kvo_pool *s) {
     memcpy(p->ring, s->ring, (size_t)s->NB * sizeof(int32_t));
     memcpy(p->table, s->table, (size_t)s->max_ctx * s->max_blk * sizeof(int32_t));
     memcpy(p->len, s->len, (size_t)s->max_ctx * sizeof(int64_t));
+    memcpy(p->reuse, s->reuse, (size_t)s->max_ctx * sizeof(int64_t));
+    memcpy(p->last_access, s->last_access, (size_t)s->max_ctx * sizeof(int64_t));
+    p->clock = s->clock;
     p->head = s->head; p->tail = s->tail;
     p->peak_live = s->peak_live; p->cow_count = s->cow_count; p->rows_copied = s->rows_copied;
     return p;
@@ -192,6 +207,8 @@ int kvo_import(kvo_pool *p, const void *buf, int64_t n, int32_t *out_ctx) {
     for (int64_t j = 0; j < nblk(p, n); ++j) t[j] = alloc_block(p);
     for (int64_t tok = 0; tok < n; ++tok) store_token(p, t, tok, buf, n, tok);
     p->len[c] = n;
+    p->clock += 1;
+    born(p, c);
     *out_ctx = c;
     return KVO_OK;
 }
@@ -217,6 +234,8 @@ int kvo_materialize(kvo_pool *p, int32_t c, int64_t t0, int64_t t1, void *dst, i
                        (size_t)p->row);
                 p->rows_copied += 1;
             }
+    p->clock += 1;
+    read_by_other(p, c);
     return KVO_OK;
 }
 
@@ -232,6 +251,8 @@ int kvo_fork(kvo_pool *p, int32_t parent, int32_t k, int32_t *out_children) {
     for (int32_t c = 0; c < p->max_ctx; ++c) free_slots += p->len[c] < 0;
     if (free_slots < k) return KVO_OOM_CTX;
     int64_t nb = nblk(p, p->len[parent]);
+    p->clock += 1;
+    read_by_other(p, parent);
     for (int32_t j = 0; j < k; ++j) {
         int32_t c = smallest_free_ctx(p);
         for (int64_t q = 0; q < nb; ++q) {
@@ -239,6 +260,7 @@ int kvo_fork(kvo_pool *p, int32_t parent, int32_t k, int32_t *out_children) {
             p->refcount[tbl(p, parent)[q]] += 1;
         }
         p->len[c] = p->len[parent];
+        born(p, c);
         out_children[j] = c;
     }
     return KVO_OK;
@@ -293,7 +315,11 @@ int kvo_append(kvo_pool *p, int32_t n, const int32_t *ctxs, const int32_t *n_new
     }
     free(rc);
     if (free_blocks(p) < need) return KVO_OOM_BLOCKS;
-    for (int32_t i = 0; i < n; ++i) append_one(p, ctxs[i], src[i], n_new[i]);
+    p->clock += 1;
+    for (int32_t i = 0; i < n; ++i) {
+        append_one(p, ctxs[i], src[i], n_new[i]);
+        p->last_access[ctxs[i]] = p->clock;
+    }
     return KVO_OK;
 }
 
@@ -324,6 +350,8 @@ int kvo_compose(kvo_pool *p, int32_t m, const int32_t *segs, uint32_t flags, int
     if (c < 0) return KVO_OOM_CTX;
     if (free_blocks(p) < need) return KVO_OOM_BLOCKS;
 
+    p->clock += 1;
+    for (int32_t i = 0; i < m; ++i) read_by_other(p, segs[i]);
     int32_t *nt = tbl(p, c);
     int64_t cnt = 0; /* entries of the new table so far */
     off = 0;
@@ -354,6 +382,7 @@ int kvo_compose(kvo_pool *p, int32_t m, const int32_t *segs, uint32_t flags, int
         off += T;
     }
     p->len[c] = off;
+    born(p, c);
     *out_ctx = c;
     return KVO_OK;
 }
@@ -370,10 +399,57 @@ int kvo_evict(kvo_pool *p, int32_t n, const int32_t *ctxs) {
     for (int32_t i = 0; i < n; ++i)
         if (!live(p, ctxs[i])) return KVO_BAD_CTX;
     if (has_duplicates(ctxs, n)) return KVO_INVALID_ARG;
+    p->clock += 1;
     for (int32_t i = 0; i < n; ++i) {
         int32_t c = ctxs[i];
         for (int64_t j = 0; j < nblk(p, p->len[c]); ++j) release_block(p, tbl(p, c)[j]);
         p->len[c] = -1;
+    }
+    return KVO_OK;
+}
+
+/* Alg. "KV-Evict", the whole loop: score(S) = alpha * reuse(S) - beta * size(S) - gamma * age(S) for
+ * every live state, size in blocks, age = clock - last_access with the clock of this call; while the
+ * allocated blocks exceed the budget, the state with the lowest score (ties: smallest handle) is
+ * evicted by the release rule above.  Scores are computed once, before the loop, in double
+ * precision with one rounding per operation, (alpha*reuse - beta*size) - gamma*age.
+ * out_victims (cap >= number of live states) receives the evicted handles in eviction order. */
+int kvo_evict_to_budget(kvo_pool *p, double alpha, double beta, double gamma, int64_t budget_blocks,
+                        int32_t *out_victims, int32_t cap, int32_t *n_victims) {
+    if (!out_victims || !n_victims || budget_blocks < 0) return KVO_INVALID_ARG;
+    int32_t live_ctx = 0;
+    for (int32_t c = 0; c < p->max_ctx; ++c) live_ctx += p->len[c] >= 0;
+    if (cap < live_ctx) return KVO_INVALID_ARG;
+    p->clock += 1;
+    double *score = (double *)malloc((size_t)p->max_ctx * sizeof(double));
+    for (int32_t c = 0; c < p->max_ctx; ++c) {
+        if (p->len[c] < 0) continue;
+        double t1 = alpha * (double)p->reuse[c];
+        double t2 = beta * (double)nblk(p, p->len[c]);
+        double t3 = gamma * (double)(p->clock - p->last_access[c]);
+        score[c] = (t1 - t2) - t3;
+    }
+    int32_t nv = 0;
+    while (p->NB - free_blocks(p) > budget_blocks) {
+        int32_t best = -1;
+        for (int32_t c = 0; c < p->max_ctx; ++c)
+            if (p->len[c] >= 0 && (best < 0 || score[c] < score[best])) best = c;
+        if (best < 0) break;
+        for (int64_t j = 0; j < nblk(p, p->len[best]); ++j) release_block(p, tbl(p, best)[j]);
+        p->len[best] = -1;
+        out_victims[nv++] = best;
+    }
+    free(score);
+    *n_victims = nv;
+    return KVO_OK;
+}
+
+/* catalog read-out: out[0] = clock; per handle reuse and last_access (-1 for a free handle) */
+int kvo_get_catalog(const kvo_pool *p, int64_t *clock, int64_t *reuse, int64_t *last_access) {
+    *clock = p->clock;
+    for (int32_t c = 0; c < p->max_ctx; ++c) {
+        reuse[c] = p->len[c] >= 0 ? p->reuse[c] : -1;
+        last_access[c] = p->len[c] >= 0 ? p->last_access[c] : -1;
     }
     return KVO_OK;
 }

@@ -26,7 +26,7 @@ def build(force: bool = False) -> str:
     """Compile the C oracle (plain gcc -O2, one translation unit)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-fPIC", "-shared", _SRC, "-o", _LIB]
+            ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-Wall", "-Wextra", "-fPIC", "-shared", _SRC, "-o", _LIB]
         )
     return _LIB
 
@@ -58,6 +58,8 @@ def lib():
         L.kvo_get_refcounts.argtypes = [vp, p32]
         L.kvo_get_free_list.argtypes = [vp, p32, p32]
         L.kvo_stats.argtypes = [vp, p64]
+        L.kvo_evict_to_budget.argtypes = [vp, C.c_double, C.c_double, C.c_double, i64, p32, i32, p32]
+        L.kvo_get_catalog.argtypes = [vp, p64, p64, p64]
         _lib = L
     return _lib
 
@@ -149,6 +151,21 @@ class PagedOracle:
         _, cp = _i32arr(ctxs)
         st = lib().kvo_evict(self.h, len(ctxs), cp)
         return st, None
+
+    def evict_to_budget(self, alpha, beta, gamma, budget_blocks):
+        out = np.full(self.max_ctx, -1, dtype=np.int32)
+        nv = C.c_int32(0)
+        st = lib().kvo_evict_to_budget(self.h, alpha, beta, gamma, budget_blocks,
+                                       out.ctypes.data_as(C.POINTER(C.c_int32)), self.max_ctx, C.byref(nv))
+        return st, (out[: nv.value].tolist() if st == OK else None)
+
+    def catalog(self):
+        clock = C.c_int64(0)
+        reuse = np.empty(self.max_ctx, dtype=np.int64)
+        last = np.empty(self.max_ctx, dtype=np.int64)
+        lib().kvo_get_catalog(self.h, C.byref(clock), reuse.ctypes.data_as(C.POINTER(C.c_int64)),
+                              last.ctypes.data_as(C.POINTER(C.c_int64)))
+        return {"clock": clock.value, "reuse": reuse.tolist(), "last_access": last.tolist()}
 
     # -- introspection ----------------------------------------------------
     def ctx_len(self, c: int):

@@ -482,3 +482,107 @@ def test_random_walks_match_value_model(seed):
         check_conservation(snapshot(o), NB, BS_BF)
         check_against_value_model(o, vm, L_BF, ROW_BF)
     assert ok > 15
+
+
+# ---------------------------------------------------------------- Alg. KV-Evict: score and budget loop
+
+
+def _busy_pool(seed=21):
+    """A pool with shared, forked, appended, composed contexts and a spread of reuse / age / size."""
+    rng = np.random.default_rng(seed)
+    o = small_pool(NB=64, BS=4, max_ctx=12, max_blk=32, order=rng.permutation(64))
+    a = o.imp(rand_buf(rng, o, 10), 10)[1]
+    b = o.imp(rand_buf(rng, o, 23), 23)[1]
+    kids = o.fork(a, 3)[1]
+    o.append([kids[0]], [5], [rand_buf(rng, o, 5)])
+    o.materialize(b, 0, 23)
+    o.materialize(b, 3, 9)
+    z = o.compose([kids[1], b])[1]
+    o.append([kids[2]], [9], [rand_buf(rng, o, 9)])
+    o.materialize(kids[0], 0, 15)
+    return o, rng
+
+
+def test_catalog_counts_reads_and_stamps_the_clock():
+    o, _ = _busy_pool()
+    cat = o.catalog()
+    # operators so far: import a(1) import b(2) fork(3) append(4) materialize b(5,6) compose(7) append(8) materialize(9)
+    assert cat["clock"] == 9
+    # handles: a=0 b=1 kids=2,3,4 z=5
+    assert cat["reuse"][:6] == [1, 3, 1, 1, 0, 0]          # a: fork; b: 2 materialize + compose; k0: materialize; k1: compose
+    assert cat["last_access"][:6] == [3, 7, 9, 7, 8, 7]
+    assert cat["reuse"][6] == -1 and cat["last_access"][6] == -1
+
+
+def _evict_in_order_until(o, order, budget):
+    victims = []
+    for c in order:
+        if o.stats()["live_blocks"] <= budget:
+            break
+        assert o.evict([c])[0] == 0
+        victims.append(c)
+    return victims
+
+
+@pytest.mark.parametrize("budget", [0, 5, 9, 14, 1000])
+def test_age_only_score_is_lru(budget):
+    o, _ = _busy_pool()
+    ref = o.clone()
+    cat = o.catalog()
+    live = o.live_ctxs()
+    lru_order = sorted(live, key=lambda c: (cat["last_access"][c], c))  # oldest first: largest age, lowest score
+    st, victims = o.evict_to_budget(0.0, 0.0, 1.0, budget)
+    assert st == 0
+    assert victims == _evict_in_order_until(ref, lru_order, budget)
+    a, b = snapshot(o), snapshot(ref)
+    assert a == b and np.array_equal(o.pool_view(), ref.pool_view())
+    check_conservation(a, o.NB, o.BS)
+    if budget == 1000:
+        assert victims == []
+    if budget == 0:
+        assert sorted(victims) == sorted(live) and sorted(o.free_list().tolist()) == list(range(o.NB))
+
+
+def test_size_only_and_reuse_only_scores():
+    o, _ = _busy_pool()
+    ref = o.clone()
+    live = o.live_ctxs()
+    by_size = sorted(live, key=lambda c: (-(-(-o.ctx_len(c) // o.BS)), c))  # most blocks first
+    st, victims = o.evict_to_budget(0.0, 1.0, 0.0, 6)
+    assert victims == _evict_in_order_until(ref, by_size, 6) and snapshot(o) == snapshot(ref)
+    o, _ = _busy_pool()
+    ref = o.clone()
+    cat = o.catalog()
+    by_reuse = sorted(o.live_ctxs(), key=lambda c: (cat["reuse"][c], c))  # least reused first
+    st, victims = o.evict_to_budget(1.0, 0.0, 0.0, 6)
+    assert victims == _evict_in_order_until(ref, by_reuse, 6) and snapshot(o) == snapshot(ref)
+
+
+@pytest.mark.parametrize("weights", [(1.5, 0.25, 0.1), (0.3, 2.0, 0.7), (10.0, 0.01, 3.3)])
+def test_mixed_score_orders_victims_by_the_formula(weights):
+    al, be, ga = weights
+    o, _ = _busy_pool()
+    ref = o.clone()
+    cat = o.catalog()
+    clock = cat["clock"] + 1  # the eviction call itself advances the clock before ages are taken
+    score = {c: (al * cat["reuse"][c] - be * (-(-o.ctx_len(c) // o.BS))) - ga * (clock - cat["last_access"][c])
+             for c in o.live_ctxs()}
+    order = sorted(score, key=lambda c: (score[c], c))
+    st, victims = o.evict_to_budget(al, be, ga, 7)
+    assert st == 0 and victims == _evict_in_order_until(ref, order, 7)
+    assert snapshot(o) == snapshot(ref)
+
+
+def test_shared_prefix_survives_scored_eviction():
+    rng = np.random.default_rng(5)
+    o = small_pool(NB=32, BS=4, max_ctx=8, max_blk=16)
+    p = o.imp(rand_buf(rng, o, 16), 16)[1]            # 4 blocks
+    kids = o.fork(p, 3)[1]
+    o.append(kids, [4, 4, 4], [rand_buf(rng, o, 4) for _ in kids])  # one private block each -> 7 live
+    o.materialize(p, 0, 16)                           # the parent is the most recently used
+    st, victims = o.evict_to_budget(0.0, 0.0, 1.0, 5)
+    # evicting a child frees only its private block: two children go, the prefix stays with p and the third
+    assert victims == kids[:2]
+    assert o.stats()["live_blocks"] == 5
+    assert np.array_equal(o.table(p), o.table(kids[2])[:4])
+    assert o.evict_to_budget(0.0, 0.0, 1.0, -1)[0] == paged.INVALID_ARG
