@@ -362,6 +362,15 @@ def extra_report(args):
             assert be.o.sync_status() == 0
             calls = len(d.log)
             kms = sum(dms.values())
+            # scored eviction (Alg. KV-Evict on the device): halve the live blocks by LRU score
+            live0 = be.o.stats()["live_blocks"]
+            t1 = time.perf_counter()
+            st_e, victims = be.o.evict_to_budget(0.0, 0.0, 1.0, live0 // 2)
+            t_evict = time.perf_counter() - t1
+            assert st_e == 0
+            out.update({"evict_to_budget": {"live_blocks_before": live0, "budget": live0 // 2, "victims": len(victims),
+                                            "live_blocks_after": be.o.stats()["live_blocks"],
+                                            "call_ms_including_sync": 1e3 * t_evict}})
             out.update({"block_size": bs, "demand_blocks": demand, "n_blocks": nb, "pool_GiB": g.pool_bytes / 2**30,
                         "library_calls": calls, "calls_by_kind": d.counts,
                         "oom_answers": sum(1 for _, _, st in d.log if st == churn.OOM_BLOCKS),

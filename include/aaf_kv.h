@@ -193,6 +193,20 @@ int aaf_kv_compose(aaf_kv_pool *pool, int32_t m, const aaf_ctx_t *segs, uint32_t
  * array.  Errors: BAD_CTX, INVALID_ARG (duplicate), TOO_MANY. */
 int aaf_kv_evict(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, void *stream);
 
+/* evict to a budget -- Alg. "KV-Evict", the whole loop, selected on the device.  For every live
+ * context score(S) = alpha * reuse(S) - beta * size(S) - gamma * age(S): reuse = number of times S
+ * was read by materialize, fork or compose (per occurrence); size = its block-table length; age =
+ * logical clock of this call - clock of the last call that read, wrote or created S (the clock counts
+ * successful state-touching calls).  Scores are taken once, in double precision, one rounding per
+ * operation.  While the live blocks (n_blocks - free) exceed budget_blocks, the context with the
+ * lowest score (ties: smallest handle) is evicted by the release rule of aaf_kv_evict.  Shared
+ * blocks survive while another context references them.  out_victims (host, cap >= number of live
+ * contexts) receives the evicted handles in order, *n_victims their count.  The call synchronises
+ * `stream` (the host needs the victims).  alpha = beta = 0, gamma > 0 is LRU.
+ * Errors: INVALID_ARG (negative budget, non-finite weight, cap too small), CUDA. */
+int aaf_kv_evict_to_budget(aaf_kv_pool *pool, double alpha, double beta, double gamma, int64_t budget_blocks,
+                           aaf_ctx_t *out_victims, int32_t cap, int32_t *n_victims, void *stream);
+
 /* Host-buffer forms of the transfer pack / unpack (the device end of Sec. 5.4's transport when
  * the peer is host memory).  staging_dev (device, >= n * bpt bytes) is caller-owned scratch.
  * materialize_host gathers into staging_dev and copies it to dst_host; import_host copies
@@ -232,6 +246,8 @@ int aaf_kv_ctx_len(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t *n_tokens);
 int aaf_kv_get_table(aaf_kv_pool *pool, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks);
 int aaf_kv_get_refcounts(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */);
 int aaf_kv_get_free_list(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */, int32_t *n_free);
+/* Catalog counters per handle (max_ctx entries each; -1 for a free handle) and the logical clock. */
+int aaf_kv_get_catalog(aaf_kv_pool *pool, int64_t *clock, int64_t *reuse_out, int64_t *last_access_out);
 int aaf_kv_pool_stats(aaf_kv_pool *pool, aaf_kv_stats *out);
 /* Returns the sticky device status (AAF_OK, AAF_ERR_CORRUPT or AAF_ERR_TIMEOUT) and clears it. */
 int aaf_kv_sync_status(aaf_kv_pool *pool);

@@ -74,6 +74,8 @@ SYMBOLS = {
     "aaf_kv_materialize_host_chunked": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, _i32, C.POINTER(C.c_uint32),
                                                   _i32, _p32, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host_chunked": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _i32, _p32, _vp]),
+    "aaf_kv_evict_to_budget": (C.c_int, [_vp, C.c_double, C.c_double, C.c_double, _i64, _p32, _i32, _p32, _vp]),
+    "aaf_kv_get_catalog": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
     "aaf_kv_ctx_len": (C.c_int, [_vp, _i32, C.POINTER(_i64)]),
     "aaf_kv_get_table": (C.c_int, [_vp, _i32, _p32, _i32, _p32]),
     "aaf_kv_get_refcounts": (C.c_int, [_vp, _p32]),
@@ -133,6 +135,9 @@ def aaf_kv_materialize_host_chunked(pool, ctx, t0, t1, dst_host, dst_bytes, stag
                                                   chunk_tokens, done_flags, flags_cap, n_chunks_out, out_desc, stream)
 def aaf_kv_import_host_chunked(pool, src_host, desc, staging, staging_bytes, chunk_tokens, out_ctx, stream):
     return _fn("aaf_kv_import_host_chunked")(pool, src_host, desc, staging, staging_bytes, chunk_tokens, out_ctx, stream)
+def aaf_kv_evict_to_budget(pool, alpha, beta, gamma, budget, out_victims, cap, n_victims, stream):
+    return _fn("aaf_kv_evict_to_budget")(pool, alpha, beta, gamma, budget, out_victims, cap, n_victims, stream)
+def aaf_kv_get_catalog(pool, clock, reuse, last): return _fn("aaf_kv_get_catalog")(pool, clock, reuse, last)
 def aaf_kv_ctx_len(pool, ctx, out): return _fn("aaf_kv_ctx_len")(pool, ctx, out)
 def aaf_kv_get_table(pool, ctx, out, cap, n_blocks): return _fn("aaf_kv_get_table")(pool, ctx, out, cap, n_blocks)
 def aaf_kv_get_refcounts(pool, out): return _fn("aaf_kv_get_refcounts")(pool, out)
@@ -278,6 +283,25 @@ class KVPool:
         st = aaf_kv_import_host(self.h, src_host.data_ptr(), C.byref(xd), staging.data_ptr(),
                                 staging.numel() * staging.element_size(), C.byref(out), self._stream())
         return st, (out.value if st == AAF_OK else None)
+
+    def evict_to_budget(self, alpha, beta, gamma, budget_blocks):
+        out = (C.c_int32 * self.max_ctx)()
+        nv = C.c_int32(0)
+        st = aaf_kv_evict_to_budget(self.h, alpha, beta, gamma, budget_blocks, out, self.max_ctx, C.byref(nv),
+                                    self._stream())
+        return st, (list(out[: nv.value]) if st == AAF_OK else None)
+
+    def catalog(self):
+        import numpy as np
+
+        clock = C.c_int64(0)
+        reuse = np.empty(self.max_ctx, dtype=np.int64)
+        last = np.empty(self.max_ctx, dtype=np.int64)
+        st = aaf_kv_get_catalog(self.h, C.byref(clock), reuse.ctypes.data_as(C.POINTER(C.c_int64)),
+                                last.ctypes.data_as(C.POINTER(C.c_int64)))
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        return {"clock": clock.value, "reuse": reuse.tolist(), "last_access": last.tolist()}
 
     def materialize_host_chunked(self, ctx, t0, t1, dst_host, staging, chunk_tokens, flags=None):
         """flags: pinned torch int32 tensor receiving one completion flag per chunk (or None)."""

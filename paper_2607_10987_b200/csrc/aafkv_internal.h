@@ -52,6 +52,11 @@ struct DevState {
     int *tables;     // [max_ctx][max_blk]
     Piece *pieces;   // [max_pieces]
     int *scratch;    // [3 * max_batch] per-batch scratch of the append planner
+    // metadata catalog per handle (App. A.2): tokens (-1 = free handle), reads by other states, last access
+    long long *cat_len;
+    unsigned long long *cat_reuse;
+    long long *cat_last;
+    double *cat_score;  // scratch of the scored eviction
 };
 
 // ---- per-call argument records (written by the host into pinned memory, read by planners)
@@ -81,18 +86,24 @@ struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
 };
 
 // ---- launchers (each returns cudaGetLastError() of its launches)
+// `clock` is the logical clock of the call (count of successful state-touching calls); planners stamp
+// it into the catalog.  A DevState without catalog arrays (cat_len == nullptr) skips the stamping.
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
-                                    cudaStream_t st);
+                                    long long clock, cudaStream_t st);
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
-                               cudaStream_t st);
-cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, int nblk, int k, const int *children_dev,
-                        cudaStream_t st);
+                               long long clock, cudaStream_t st);
+cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
+                        long long clock, cudaStream_t st);
 cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
-                               int total_slots, int max_batch, int dry_run, cudaStream_t st);
+                               int total_slots, int max_batch, int dry_run, long long clock, cudaStream_t st);
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
-                                int total_fresh, int total_slots, int out_ctx, cudaStream_t st);
+                                int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st);
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
                          cudaStream_t st);
+// Scored eviction (Alg. KV-Evict): result[0] = number of victims, result[1] = free blocks afterwards,
+// result[2..] = victims in eviction order; `result` is host memory the device can write.
+cudaError_t launch_evict_to_budget(const Geom &g, const DevState &s, double alpha, double beta, double gamma,
+                                   long long budget_blocks, long long clock, int *result, cudaStream_t st);
 // launch shapes of the copy engines for one pool geometry (see copy_tuning_init)
 struct CopyTuning {
     int bulk_chunk, bulk_stages, bulk_ctas, bulk_l2;

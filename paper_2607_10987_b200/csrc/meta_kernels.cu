@@ -101,7 +101,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *total) {
 // ------------------------------------------------------------------------------------------
 // materialize: one piece per block of the token range
 __global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState s, int ctx, long long t0,
-                                                               long long t1, char *dst) {
+                                                               long long t1, char *dst, long long clock) {
     const long long j0 = t0 / g.BS, j1 = (t1 - 1) / g.BS;
     const long long n = t1 - t0;
     const int *table = s.tables + (long long)ctx * g.max_blk;
@@ -111,13 +111,19 @@ __global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState 
         s.pieces[j - j0] = make_piece(pool_slot(g, b, lo - j * g.BS), g.layer_stride, g.run, dst + (lo - t0) * g.row,
                                       2 * n * g.row, n * g.row, (unsigned)((hi - lo) * g.row));
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(n * 2 * g.L * g.row));
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(n * 2 * g.L * g.row));
+        if (s.cat_len) {  // the state was read by a transfer
+            s.cat_reuse[ctx] += 1;
+            s.cat_last[ctx] = clock;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------
 // import: reserve ceil(n / BS) ring entries in order, write the table, one piece per block
 __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevState s, int ctx, long long n,
-                                                                   const char *src) {
+                                                                   const char *src, long long clock) {
     const int nblk = (int)((n + g.BS - 1) / g.BS);
     const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
     const bool ok = (tail - head0) >= (unsigned long long)nblk;
@@ -142,14 +148,20 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevSt
             s.ctl->head = head0 + nblk;
             note_alloc(s.ctl, g, head0 + nblk, tail);
             s.ctl->payload_bytes += (unsigned long long)(n * 2 * g.L * g.row);
+            if (s.cat_len) {
+                s.cat_len[ctx] = n;
+                s.cat_reuse[ctx] = 0;
+                s.cat_last[ctx] = clock;
+            }
         }
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // fork: k table copies, refcount += k per parent entry
-__global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int parent, int nblk, int k,
-                                                   const int *__restrict__ children_host) {
+__global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int parent, long long T, int k,
+                                                   const int *__restrict__ children_host, long long clock) {
+    const int nblk = (int)((T + g.BS - 1) / g.BS);
     __shared__ int sh_children[1024];
     const int *children = stage_args(children_host, k, sh_children, 1024);
     const int *pt = s.tables + (long long)parent * g.max_blk;
@@ -160,6 +172,15 @@ __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int paren
         const int b = pt[j];
         s.tables[(long long)children[q] * g.max_blk + j] = b;
         if (q == 0) atomicAdd(&s.refcount[b], k);
+        if (j == 0 && s.cat_len) {  // catalog: the child is born, the parent was read
+            s.cat_len[children[q]] = T;
+            s.cat_reuse[children[q]] = 0;
+            s.cat_last[children[q]] = clock;
+            if (q == 0) {
+                s.cat_reuse[parent] += 1;
+                s.cat_last[parent] = clock;
+            }
+        }
     }
 }
 
@@ -175,7 +196,8 @@ __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int paren
 // scratch layout (ints): tailb[n] | need[n] | alloc_off[n]
 __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevState s,
                                                                    const AppendEntry *__restrict__ ent_host, int n,
-                                                                   int total_slots, int max_batch, int dry_run) {
+                                                                   int total_slots, int max_batch, int dry_run,
+                                                                   long long clock) {
     __shared__ AppendEntry sh_ent[768];
     const AppendEntry *ent = stage_args(ent_host, n, sh_ent, 768);
     int *tailb = s.scratch;
@@ -276,6 +298,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
                                   (unsigned)((thi - tlo) * g.row));
         atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((thi - tlo) * g.row * 2 * g.L));
     }
+    if (ok && s.cat_len)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            s.cat_len[ent[i].ctx] = ent[i].T + ent[i].n_new;
+            s.cat_last[ent[i].ctx] = clock;
+        }
     __syncthreads();
     if (threadIdx.x == 0) {
         if (!ok) {
@@ -298,7 +325,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
                                                                     const ComposeSeg *__restrict__ segs_host, int m,
                                                                     int total_work, int total_fresh, int total_slots,
-                                                                    int out_ctx) {
+                                                                    int out_ctx, long long clock) {
     __shared__ ComposeSeg sh_segs[512];
     const ComposeSeg *segs = stage_args(segs_host, m, sh_segs, 512);
     const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
@@ -358,6 +385,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
             atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((s_hi - s_lo) * g.row * 2 * g.L));
         }
     }
+    if (ok && s.cat_len)
+        for (int i = threadIdx.x; i < m; i += blockDim.x) {  // every occurrence of a segment is one read
+            atomicAdd(&s.cat_reuse[segs[i].ctx], 1ull);
+            s.cat_last[segs[i].ctx] = clock;
+        }
     __syncthreads();
     if (threadIdx.x == 0) {
         if (!ok) {
@@ -365,6 +397,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
         } else {
             s.ctl->head = head0 + total_fresh;
             note_alloc(s.ctl, g, head0 + total_fresh, tail);
+            if (s.cat_len) {
+                s.cat_len[out_ctx] = segs[m - 1].off + segs[m - 1].T;
+                s.cat_reuse[out_ctx] = 0;
+                s.cat_last[out_ctx] = clock;
+            }
         }
     }
 }
@@ -460,9 +497,109 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevSta
     // every flag has been taken: clear the scratch marks of the touched blocks
     for (int e = threadIdx.x; e < total; e += blockDim.x)
         s.last_pos[evict_entry_block(g, s, ctx, ent_off, n, e)] = -1;
+    if (s.cat_len)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) s.cat_len[ctx[i]] = -1;
     if (threadIdx.x == 0) {
         if (tail0 + carry - s.ctl->head > (unsigned long long)g.NB) set_status(s.ctl, AAF_ERR_CORRUPT, 8);
         s.ctl->tail = tail0 + carry;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// scored eviction (Alg. KV-Evict, the whole loop) in one CTA
+//   score(S) = alpha * reuse(S) - beta * size(S) - gamma * age(S), size in blocks, age = clock - last access,
+//   computed once in double precision with one rounding per operation (no fused multiply-add), so that
+//   the victim order is the same on any IEEE machine.  While the live blocks exceed the budget the
+//   state with the lowest score (ties: smallest handle) is released entry by entry with the same
+//   rules as evict: a block is freed at its last occurrence in the victim's table, in table order.
+__global__ void __launch_bounds__(PLAN_THREADS) evict_to_budget_kernel(Geom g, DevState s, double alpha, double beta,
+                                                                       double gamma, long long budget,
+                                                                       long long clock, int *result) {
+    __shared__ double sh_score[32];
+    __shared__ int sh_id[32];
+    __shared__ int sh_victim;
+    __shared__ long long sh_live;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int c = threadIdx.x; c < g.max_ctx; c += blockDim.x) {
+        const long long len = s.cat_len[c];
+        if (len < 0) continue;
+        const double t1 = __dmul_rn(alpha, (double)s.cat_reuse[c]);
+        const double t2 = __dmul_rn(beta, (double)((len + g.BS - 1) / g.BS));
+        const double t3 = __dmul_rn(gamma, (double)(clock - s.cat_last[c]));
+        s.cat_score[c] = __dsub_rn(__dsub_rn(t1, t2), t3);
+    }
+    if (threadIdx.x == 0) sh_live = (long long)g.NB - (long long)(s.ctl->tail - s.ctl->head);
+    __syncthreads();
+    int nv = 0;
+    while (true) {
+        if (sh_live <= budget) break;  // uniform: read after a barrier
+        // lowest (score, handle) among the live states
+        double best = 0.0;
+        int best_id = -1;
+        for (int c = threadIdx.x; c < g.max_ctx; c += blockDim.x) {
+            if (s.cat_len[c] < 0) continue;
+            const double sc = s.cat_score[c];
+            if (best_id < 0 || sc < best) { best = sc; best_id = c; }  // ascending c: ties keep the smaller handle
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            const double os = __shfl_down_sync(0xffffffffu, best, d);
+            const int oi = __shfl_down_sync(0xffffffffu, best_id, d);
+            if (oi >= 0 && (best_id < 0 || os < best || (os == best && oi < best_id))) { best = os; best_id = oi; }
+        }
+        if (lane == 0) { sh_score[wid] = best; sh_id[wid] = best_id; }
+        __syncthreads();
+        if (wid == 0) {
+            best = sh_score[lane];
+            best_id = sh_id[lane];
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                const double os = __shfl_down_sync(0xffffffffu, best, d);
+                const int oi = __shfl_down_sync(0xffffffffu, best_id, d);
+                if (oi >= 0 && (best_id < 0 || os < best || (os == best && oi < best_id))) { best = os; best_id = oi; }
+            }
+            if (lane == 0) sh_victim = best_id;
+        }
+        __syncthreads();
+        const int v = sh_victim;
+        if (v < 0) break;
+        // release the victim's entries
+        const int nb = (int)((s.cat_len[v] + g.BS - 1) / g.BS);
+        const int *table = s.tables + (long long)v * g.max_blk;
+        for (int e = threadIdx.x; e < nb; e += blockDim.x) {
+            const int b = table[e];
+            if (atomicSub(&s.refcount[b], 1) <= 0) set_status(s.ctl, AAF_ERR_CORRUPT, 9);
+            atomicMax(&s.last_pos[b], e);
+        }
+        __syncthreads();
+        const unsigned long long tail0 = s.ctl->tail;
+        int carry = 0;
+        for (int base = 0; base < nb; base += blockDim.x) {
+            const int e = base + threadIdx.x;
+            int b = -1, flag = 0;
+            if (e < nb) {
+                b = table[e];
+                flag = (s.refcount[b] == 0 && s.last_pos[b] == e);
+            }
+            int tot;
+            const int ex = block_exclusive_scan(flag, &tot);
+            if (flag) s.ring[(tail0 + (unsigned long long)(carry + ex)) % (unsigned long long)g.NB] = b;
+            carry += tot;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < nb; e += blockDim.x) s.last_pos[table[e]] = -1;
+        if (threadIdx.x == 0) {
+            s.ctl->tail = tail0 + carry;
+            sh_live -= carry;
+            s.cat_len[v] = -1;
+            result[2 + nv] = v;
+        }
+        ++nv;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        result[0] = nv;
+        result[1] = (int)(s.ctl->tail - s.ctl->head);
     }
 }
 
@@ -477,29 +614,31 @@ static int grid_for(long long items, int threads, int cap) {
 }
 
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
-                                    cudaStream_t st) {
+                                    long long clock, cudaStream_t st) {
     const long long nb = (t1 - 1) / g.BS - t0 / g.BS + 1;
-    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst);
+    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
-                               cudaStream_t st) {
-    plan_import_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, ctx, n, src);
+                               long long clock, cudaStream_t st) {
+    plan_import_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, ctx, n, src, clock);
     return cudaGetLastError();
 }
-cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, int nblk, int k, const int *children_dev,
-                        cudaStream_t st) {
-    fork_kernel<<<grid_for((long long)nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, nblk, k, children_dev);
+cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
+                        long long clock, cudaStream_t st) {
+    const long long nblk = (T + g.BS - 1) / g.BS;
+    fork_kernel<<<grid_for(nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, T, k, children_dev, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
-                               int total_slots, int max_batch, int dry_run, cudaStream_t st) {
-    plan_append_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, entries_dev, n, total_slots, max_batch, dry_run);
+                               int total_slots, int max_batch, int dry_run, long long clock, cudaStream_t st) {
+    plan_append_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, entries_dev, n, total_slots, max_batch, dry_run, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
-                                int total_fresh, int total_slots, int out_ctx, cudaStream_t st) {
-    plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, m, total_work, total_fresh, total_slots, out_ctx);
+                                int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st) {
+    plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, m, total_work, total_fresh, total_slots, out_ctx,
+                                                    clock);
     return cudaGetLastError();
 }
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
@@ -508,6 +647,12 @@ cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_evict_to_budget(const Geom &g, const DevState &s, double alpha, double beta, double gamma,
+                                   long long budget_blocks, long long clock, int *result, cudaStream_t st) {
+    evict_to_budget_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, alpha, beta, gamma, budget_blocks, clock, result);
     return cudaGetLastError();
 }
 

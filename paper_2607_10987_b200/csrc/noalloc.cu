@@ -109,7 +109,7 @@ extern "C" int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t laye
     s.ctl = &sc->ctl;
     s.tables = sc->table - j0;  // the planner indexes the table by absolute block position
     s.pieces = sc->pieces;
-    if (launch_plan_materialize(g, s, 0, tok_begin, tok_end, static_cast<char *>(dst_dev), st) != cudaSuccess)
+    if (launch_plan_materialize(g, s, 0, tok_begin, tok_end, static_cast<char *>(dst_dev), 0, st) != cudaSuccess)
         return AAF_ERR_CUDA;
     if (launch_copy(AAF_ENGINE_VEC, g_tuning[dev], g, s, (int)nb, 0, 2 * n_layers, run, g_sm_count[dev], st) !=
         cudaSuccess)

@@ -25,7 +25,7 @@ namespace {
 constexpr int ARG_SLOTS = 16;
 
 struct Layout {
-    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, total;
+    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, total;
     int max_pieces, max_batch;
 };
 
@@ -54,6 +54,10 @@ Layout make_layout(const aaf_kv_pool_desc *d) {
     L.tables = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx * d->max_blocks_per_ctx, 256);
     L.pieces = off; off = align_up(off + sizeof(Piece) * (size_t)L.max_pieces, 256);
     L.scratch = off; off = align_up(off + sizeof(int) * 3 * (size_t)L.max_batch, 256);
+    L.cat_len = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
+    L.cat_reuse = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
+    L.cat_last = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
+    L.cat_score = off; off = align_up(off + sizeof(double) * (size_t)d->max_ctx, 256);
     L.total = off;
     return L;
 }
@@ -86,6 +90,8 @@ struct aaf_kv_pool {
     std::vector<long long> len;  // tokens per handle, -1 = free
     int live_ctx = 0;
     long long free_lb = 0;       // guaranteed lower bound of the device's free-block count
+    long long clock = 0;         // logical clock: successful state-touching calls so far
+    int *result = nullptr;       // pinned, device-writable: result of the scored eviction (max_ctx + 2 ints)
     cudaStream_t last_stream = nullptr;
     // pinned argument ring
     char *args = nullptr;
@@ -224,8 +230,10 @@ int materialize_impl(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void
     const long long n = t1 - t0;
     if ((unsigned long long)dst_bytes < (unsigned long long)(n * bpt_of(p))) return AAF_ERR_DST_TOO_SMALL;
     p->last_stream = st;
-    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(dst_dev), st) != cudaSuccess)
+    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(dst_dev), p->clock + 1, st) !=
+        cudaSuccess)
         return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     const int n_slots = (int)((t1 - 1) / p->g.BS - t0 / p->g.BS + 1);
     const int rc = run_copy(p, AAF_OP_MATERIALIZE, n_slots, n, st);
@@ -251,8 +259,9 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
                             st) != cudaSuccess)
             return AAF_ERR_CUDA;
     }
-    if (launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(src_dev), st) != cudaSuccess)
+    if (launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(src_dev), p->clock + 1, st) != cudaSuccess)
         return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= nb;
     p->len[c] = n;
@@ -343,6 +352,10 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     p->s.tables = reinterpret_cast<int *>(ws + lay.tables);
     p->s.pieces = reinterpret_cast<Piece *>(ws + lay.pieces);
     p->s.scratch = reinterpret_cast<int *>(ws + lay.scratch);
+    p->s.cat_len = reinterpret_cast<long long *>(ws + lay.cat_len);
+    p->s.cat_reuse = reinterpret_cast<unsigned long long *>(ws + lay.cat_reuse);
+    p->s.cat_last = reinterpret_cast<long long *>(ws + lay.cat_last);
+    p->s.cat_score = reinterpret_cast<double *>(ws + lay.cat_score);
     p->len.assign((size_t)desc->max_ctx, -1);
     p->free_lb = desc->n_blocks;
 
@@ -353,6 +366,8 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
                    cudaSuccess;
     for (int i = 0; ok && i < ARG_SLOTS; ++i)
         ok = cudaEventCreateWithFlags(&p->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaHostAlloc(reinterpret_cast<void **>(&p->result), sizeof(int) * ((size_t)desc->max_ctx + 2),
+                             cudaHostAllocMapped) == cudaSuccess;
     // device state: counters, reference counts 0, ring, evict scratch -1
     DevCtl ctl;
     memset(&ctl, 0, sizeof(ctl));
@@ -362,6 +377,8 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     ok = ok && cudaMemcpy(p->s.ctl, &ctl, sizeof(ctl), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(p->s.ring, ring.data(), sizeof(int) * ring.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(p->s.last_pos, 0xff, sizeof(int) * (size_t)desc->n_blocks) == cudaSuccess;
+    ok = ok && cudaMemset(p->s.cat_len, 0xff, sizeof(long long) * (size_t)desc->max_ctx) == cudaSuccess;  // -1: free
+    ok = ok && cudaMemset(p->s.cat_reuse, 0, lay.total - lay.cat_reuse) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -389,6 +406,7 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
     for (int i = 0; i < ARG_SLOTS; ++i)
         if (p->slot_ev[i]) cudaEventDestroy(p->slot_ev[i]);
     if (p->args) cudaFreeHost(p->args);
+    if (p->result) cudaFreeHost(p->result);
     delete p;
     return AAF_OK;
 }
@@ -455,8 +473,10 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     p->last_stream = st;
     if (done_flags_host)
         for (int c = 0; c < n_chunks; ++c) done_flags_host[c] = 0;
-    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(staging_dev), st) != cudaSuccess)
+    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(staging_dev), p->clock + 1, st) !=
+        cudaSuccess)
         return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     bool ok = true;
     for (int c = 0; c < n_chunks && ok; ++c) {
@@ -506,8 +526,10 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     cudaEvent_t start = order_event(p);
     bool ok = start && cudaEventRecord(start, st) == cudaSuccess &&
               cudaStreamWaitEvent(p->xfer_stream, start, 0) == cudaSuccess;
-    ok = ok && launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(staging_dev), st) == cudaSuccess;
+    ok = ok && launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(staging_dev), p->clock + 1, st) ==
+                   cudaSuccess;
     if (!ok) return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= nb;
     p->len[c] = n;
@@ -543,9 +565,10 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
         children[j] = c;
     }
     const long long T = p->len[parent];
-    const cudaError_t e = launch_fork(p->g, p->s, parent, (int)nblk_of(p, T), k, children, st);
+    const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, children, p->clock + 1, st);
     release_args(p, st);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     for (int j = 0; j < k; ++j) {
         p->len[children[j]] = T;
@@ -601,7 +624,7 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             // the worst case does not fit: ask the planner (dry run) how many blocks the batch really
             // needs; only tail blocks that are still shared are copied
             unsigned long long need = 0;
-            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, st) != cudaSuccess ||
+            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, p->clock, st) != cudaSuccess ||
                 cudaStreamSynchronize(st) != cudaSuccess ||
                 cudaMemcpy(&need, &p->s.ctl->probe_need, sizeof(need), cudaMemcpyDeviceToHost) != cudaSuccess)
                 rc = AAF_ERR_CUDA;
@@ -615,9 +638,11 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             return rc;
         }
     }
-    const cudaError_t e = launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 0, st);
+    const cudaError_t e =
+        launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 0, p->clock + 1, st);
     release_args(p, st);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= charge;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] += n_new[i];
@@ -671,9 +696,10 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     ComposeSeg *dev_rec = reinterpret_cast<ComposeSeg *>(acquire_args(p));
     memcpy(dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
     const cudaError_t e =
-        launch_plan_compose(p->g, p->s, dev_rec, m, (int)work, (int)fresh, (int)slots, c, st);
+        launch_plan_compose(p->g, p->s, dev_rec, m, (int)work, (int)fresh, (int)slots, c, p->clock + 1, st);
     release_args(p, st);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= fresh;
     p->len[c] = off;
@@ -710,10 +736,54 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
     const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, st);
     release_args(p, st);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
+    p->clock += 1;
     p->meta_launches += 2;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] = -1;
     p->live_ctx -= n;
     return AAF_OK;  // the lower bound of the free count stays valid: evict only adds free blocks
+}
+
+int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gamma, int64_t budget_blocks,
+                           aaf_ctx_t *out_victims, int32_t cap, int32_t *n_victims, void *stream) {
+    if (!p || !out_victims || !n_victims || budget_blocks < 0) return AAF_ERR_INVALID_ARG;
+    if (!(alpha == alpha && beta == beta && gamma == gamma) || alpha - alpha != 0.0 || beta - beta != 0.0 ||
+        gamma - gamma != 0.0)
+        return AAF_ERR_INVALID_ARG;  // NaN or infinite weights
+    if (cap < p->live_ctx) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    if (launch_evict_to_budget(p->g, p->s, alpha, beta, gamma, budget_blocks, p->clock + 1, p->result, st) !=
+        cudaSuccess)
+        return AAF_ERR_CUDA;
+    p->meta_launches += 1;
+    // the victims are chosen on the device; the host mirror needs them before the next call
+    if (cudaStreamSynchronize(st) != cudaSuccess) return AAF_ERR_CUDA;
+    p->clock += 1;
+    const int nv = p->result[0];
+    for (int i = 0; i < nv; ++i) {
+        const int v = p->result[2 + i];
+        out_victims[i] = v;
+        p->len[v] = -1;
+    }
+    p->live_ctx -= nv;
+    p->free_lb = p->result[1];  // exact
+    *n_victims = nv;
+    return AAF_OK;
+}
+
+int aaf_kv_get_catalog(aaf_kv_pool *p, int64_t *clock, int64_t *reuse_out, int64_t *last_access_out) {
+    if (!p || !clock || !reuse_out || !last_access_out) return AAF_ERR_INVALID_ARG;
+    DeviceGuard guard(p->device);
+    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    const size_t nbytes = sizeof(long long) * (size_t)p->g.max_ctx;
+    if (cudaMemcpy(reuse_out, p->s.cat_reuse, nbytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(last_access_out, p->s.cat_last, nbytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return AAF_ERR_CUDA;
+    for (int c = 0; c < p->g.max_ctx; ++c)
+        if (p->len[c] < 0) reuse_out[c] = last_access_out[c] = -1;
+    *clock = p->clock;
+    return AAF_OK;
 }
 
 int aaf_kv_ctx_len(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t *n_tokens) {

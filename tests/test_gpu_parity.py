@@ -27,6 +27,7 @@ def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
     for (i, op, st_g, res_g, _), (_, _, st_c, res_c, _) in zip(replay(ops, gpu, seed), replay(ops, cpu, seed)):
         assert st_g == st_c, (i, op, st_g, st_c)
         assert gpu.snapshot() == cpu.snapshot(), (i, op)
+        assert gpu.o.catalog() == cpu.o.catalog(), (i, op)
         if op["op"] == "materialize" and st_c == 0:
             n = op["t1"] - op["t0"]
             assert np.array_equal(gpu.buf_layers(res_g, n, layers).reshape(-1), res_c), (i, op)
@@ -67,8 +68,8 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
     outcomes = []
     for i in range(n_ops):
         live = cpu.o.live_ctxs()
-        kind = str(rng.choice(["import", "fork", "append", "compose", "evict", "materialize", "roundtrip"],
-                              p=[0.16, 0.12, 0.26, 0.14, 0.12, 0.14, 0.06]))
+        kind = str(rng.choice(["import", "fork", "append", "compose", "evict", "materialize", "roundtrip", "budget"],
+                              p=[0.16, 0.12, 0.25, 0.14, 0.10, 0.13, 0.06, 0.04]))
         if not live:
             kind = "import"
         pick = lambda: int(rng.choice(live)) if rng.random() > 0.04 else int(rng.integers(0, g.max_ctx))
@@ -93,6 +94,10 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
         elif kind == "evict":
             who = [pick() for _ in range(int(rng.integers(1, 3)))]
             res = [be.evict(who) for be in both]
+        elif kind == "budget":  # scored eviction down to a random fraction of the current use
+            w = [float(x) for x in rng.choice([0.0, 0.5, 1.0, 2.25], size=3)]
+            budget = int(rng.integers(0, g.n_blocks))
+            res = [be.o.evict_to_budget(w[0], w[1], w[2], budget) for be in both]
         else:
             c = pick()
             T = cpu.o.ctx_len(c) or 4
@@ -110,6 +115,7 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
             assert r_g == r_c or kind == "roundtrip" and st_c == 0 and r_g == r_c, (i, kind, r_g, r_c)
         snap = cpu.snapshot()
         assert gpu.snapshot() == snap, (i, kind)
+        assert gpu.o.catalog() == cpu.o.catalog(), (i, kind)
         check_conservation(snap, g.n_blocks, g.block_size)
         if i % 8 == 7:
             assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view()), (i, kind)
@@ -164,3 +170,40 @@ def test_cow_stress_many_children():
     ops = configs.cow_stress_ops(context_tokens=507, n_children=256)
     gpu, cpu = lockstep(g, 5150, ops, max_batch=256)
     assert gpu.o.stats()["cow_count"] == 256  # every child copies: the parent keeps the old tail
+
+
+@pytest.mark.parametrize("weights", [(0.0, 0.0, 1.0), (0.0, 1.0, 0.0), (1.0, 0.0, 0.0), (1.5, 0.25, 0.1), (10.0, 0.01, 3.3)])
+@pytest.mark.parametrize("budget", [0, 6, 11, 400])
+def test_scored_eviction_to_budget(weights, budget):
+    """Alg. KV-Evict with the victims chosen on the device: same victims in the same order, same
+    tables / reference counts / free list as the oracle's loop."""
+    g = Geometry(2, 2, 64, 4, 2, 64, 12, 32)
+    order = configs.free_order(31, g.n_blocks)
+    gpu = GpuBackend(g, 31, free_order=order)
+    cpu = OracleBackend(g, 31, free_order=order)
+    for be in (gpu, cpu):
+        pay = lambda s, n: be.payload(31, s, n)
+        a = be.imp(pay(1, 10), 10)[1]
+        b = be.imp(pay(2, 23), 23)[1]
+        kids = be.fork(a, 3)[1]
+        assert be.append([kids[0]], [5], [pay(3, 5)])[0] == 0
+        be.materialize(b, 0, 23)
+        be.materialize(b, 3, 9)
+        z = be.compose([kids[1], b], 0)[1]
+        assert be.append([kids[2]], [9], [pay(4, 9)])[0] == 0
+        be.materialize(kids[0], 0, 15)
+        be.compose([b, b], 0)
+    assert gpu.o.catalog() == cpu.o.catalog()
+    rg = gpu.o.evict_to_budget(*weights, budget)
+    rc = cpu.o.evict_to_budget(*weights, budget)
+    assert rg == rc and rc[0] == 0
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.catalog() == cpu.o.catalog()
+    check_conservation(cpu.snapshot(), g.n_blocks, g.block_size)
+    assert gpu.o.stats()["live_blocks"] <= max(budget, 0) or not gpu.o.live_ctxs()
+    # the pool keeps working with exact free accounting afterwards
+    for be in (gpu, cpu):
+        assert be.imp(be.payload(31, 9, 30), 30)[0] == 0
+    assert gpu.snapshot() == cpu.snapshot()
+    assert gpu.o.evict_to_budget(float("nan"), 0.0, 1.0, 3)[0] == -1
+    assert gpu.o.evict_to_budget(0.0, 0.0, 1.0, -2)[0] == -1
+    assert gpu.o.sync_status() == 0
