@@ -444,6 +444,41 @@ int kvo_evict_to_budget(kvo_pool *p, double alpha, double beta, double gamma, in
     return KVO_OK;
 }
 
+/* Columnar export of the metadata catalog (App. A.2, table of catalog fields; Sec. 5.3: metadata in a
+ * columnar, zero-copy encoding).  State rows: one per live state in ascending handle order
+ * (state_id, n_tokens, reuse, last_access) plus list offsets into the block rows (offsets[i] =
+ * number of block rows of the states before i, offsets[n_states] = total); block rows: one per
+ * block-table entry (block_id, position range [pos_begin, pos_end) within the state, refcount of the
+ * block, byte address of the block's layer-0 K run relative to the pool base).  Returns the counts. */
+int kvo_export_catalog(const kvo_pool *p, int32_t *state_id, int64_t *n_tokens, int64_t *reuse,
+                       int64_t *last_access, int32_t *block_offsets, int32_t *block_id, int64_t *pos_begin,
+                       int64_t *pos_end, int32_t *refcount, int64_t *address, int32_t *n_states,
+                       int32_t *n_block_rows) {
+    int32_t ns = 0, nr = 0;
+    for (int32_t c = 0; c < p->max_ctx; ++c) {
+        if (p->len[c] < 0) continue;
+        state_id[ns] = c;
+        n_tokens[ns] = p->len[c];
+        reuse[ns] = p->reuse[c];
+        last_access[ns] = p->last_access[c];
+        block_offsets[ns] = nr;
+        for (int64_t j = 0; j < nblk(p, p->len[c]); ++j) {
+            int32_t b = tbl(p, c)[j];
+            block_id[nr] = b;
+            pos_begin[nr] = j * p->BS;
+            pos_end[nr] = (j + 1) * p->BS < p->len[c] ? (j + 1) * p->BS : p->len[c];
+            refcount[nr] = p->refcount[b];
+            address[nr] = (int64_t)b * 2 * p->BS * p->row;
+            nr += 1;
+        }
+        ns += 1;
+    }
+    block_offsets[ns] = nr;
+    *n_states = ns;
+    *n_block_rows = nr;
+    return KVO_OK;
+}
+
 /* catalog read-out: out[0] = clock; per handle reuse and last_access (-1 for a free handle) */
 int kvo_get_catalog(const kvo_pool *p, int64_t *clock, int64_t *reuse, int64_t *last_access) {
     *clock = p->clock;

@@ -586,3 +586,49 @@ def test_shared_prefix_survives_scored_eviction():
     assert o.stats()["live_blocks"] == 5
     assert np.array_equal(o.table(p), o.table(kids[2])[:4])
     assert o.evict_to_budget(0.0, 0.0, 1.0, -1)[0] == paged.INVALID_ARG
+
+
+# ---------------------------------------------------------------- columnar catalog export
+
+
+def test_catalog_export_is_an_arrow_list_of_block_rows():
+    import pyarrow as pa
+
+    o, _ = _busy_pool()
+    cols = o.export_catalog()
+    live = o.live_ctxs()
+    cat = o.catalog()
+    assert cols["state_id"].tolist() == live
+    assert cols["n_tokens"].tolist() == [o.ctx_len(c) for c in live]
+    assert cols["reuse"].tolist() == [cat["reuse"][c] for c in live]
+    assert cols["last_access"].tolist() == [cat["last_access"][c] for c in live]
+    tables = [o.table(c) for c in live]
+    # offsets = running sum of the table lengths; block ids = the tables laid end to end (library routines)
+    assert cols["block_offsets"].tolist() == [0] + np.cumsum([len(t) for t in tables]).tolist()
+    assert np.array_equal(cols["block_id"], np.concatenate(tables))
+    # the offsets and values buffers are a valid Arrow ListArray without any copy or conversion
+    lst = pa.ListArray.from_arrays(pa.array(cols["block_offsets"], type=pa.int32()),
+                                   pa.array(cols["block_id"], type=pa.int32()))
+    lst.validate(full=True)
+    assert lst.to_pylist() == [t.tolist() for t in tables]
+    # position ranges tile [0, n_tokens) of each state in steps of the block size
+    for i, c in enumerate(live):
+        a, b = cols["block_offsets"][i], cols["block_offsets"][i + 1]
+        begins, ends = cols["pos_begin"][a:b], cols["pos_end"][a:b]
+        assert begins[0] == 0 and ends[-1] == o.ctx_len(c)
+        assert np.array_equal(begins[1:], ends[:-1]) and np.all(ends - begins <= o.BS) and np.all(ends > begins)
+        assert np.all((ends - begins)[:-1] == o.BS)
+    assert np.array_equal(cols["refcount"], o.refcounts()[cols["block_id"]])
+    # the address column locates the block's rows: layer 0, K, slot 0 of block b
+    pv = o.pool_view()
+    flat = pv.reshape(-1)
+    for r in (0, len(cols["block_id"]) // 2, len(cols["block_id"]) - 1):
+        b = int(cols["block_id"][r])
+        addr = int(cols["address"][r])
+        assert np.array_equal(flat[addr:addr + o.row], pv[0, b, 0, 0])
+
+
+def test_catalog_export_of_an_empty_pool():
+    o = small_pool()
+    cols = o.export_catalog()
+    assert cols["state_id"].size == 0 and cols["block_offsets"].tolist() == [0] and cols["block_id"].size == 0
