@@ -362,6 +362,18 @@ def extra_report(args):
             assert be.o.sync_status() == 0
             calls = len(d.log)
             kms = sum(dms.values())
+            # columnar catalog export of the final state (two kernels), timed with events over 20 repeats
+            be.o.export_catalog()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                cols = be.o.export_catalog()
+            e1.record()
+            torch.cuda.synchronize()
+            out.update({"catalog_export": {"states": int(cols["state_id"].numel()),
+                                           "block_rows": int(cols["block_id"].numel()),
+                                           "ms_per_export_including_buffer_allocation": e0.elapsed_time(e1) / 20}})
             # scored eviction (Alg. KV-Evict on the device): halve the live blocks by LRU score
             live0 = be.o.stats()["live_blocks"]
             t1 = time.perf_counter()

@@ -246,6 +246,32 @@ int aaf_kv_ctx_len(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t *n_tokens);
 int aaf_kv_get_table(aaf_kv_pool *pool, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks);
 int aaf_kv_get_refcounts(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */);
 int aaf_kv_get_free_list(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */, int32_t *n_free);
+/* Columnar export of the metadata catalog (App. A.2, catalog fields; Sec. 5.3: metadata kept in a
+ * columnar, zero-copy encoding).  All columns are DEVICE buffers the caller owns; they are written
+ * by kernels on `stream` and are laid out like Arrow primitive arrays and list offsets, so a consumer
+ * can wrap them without conversion.
+ *   state rows, one per live context in ascending handle order (capacity max_ctx):
+ *     state_id int32, n_tokens int64, reuse int64, last_access int64,
+ *     block_offsets int32[n_states + 1]: list offsets into the block rows (exclusive prefix sum of
+ *     the block-table lengths; capacity max_ctx + 1)
+ *   block rows, one per block-table entry (capacity = n_block_rows of aaf_kv_catalog_rows):
+ *     block_id int32, pos_begin / pos_end int64 (token range within the context), refcount int32,
+ *     address int64 (byte offset of the block's layer-0 K run from pool_base; layer l and V follow
+ *     by + l * layer_stride_bytes and + run).
+ * model_id / config_hash (M, Theta) are pool-wide and live in the pool descriptor; lineage, device
+ * and owner are the caller's tags.  aaf_kv_catalog_rows answers from the host mirror (no sync). */
+typedef struct aaf_kv_catalog_cols {
+    int32_t *state_id;
+    int64_t *n_tokens, *reuse, *last_access;
+    int32_t *block_offsets;
+    int32_t *block_id;
+    int64_t *pos_begin, *pos_end;
+    int32_t *refcount;
+    int64_t *address;
+} aaf_kv_catalog_cols;
+int aaf_kv_catalog_rows(aaf_kv_pool *pool, int32_t *n_states, int64_t *n_block_rows);
+int aaf_kv_export_catalog(aaf_kv_pool *pool, const aaf_kv_catalog_cols *cols_dev, void *stream);
+
 /* Catalog counters per handle (max_ctx entries each; -1 for a free handle) and the logical clock. */
 int aaf_kv_get_catalog(aaf_kv_pool *pool, int64_t *clock, int64_t *reuse_out, int64_t *last_access_out);
 int aaf_kv_pool_stats(aaf_kv_pool *pool, aaf_kv_stats *out);

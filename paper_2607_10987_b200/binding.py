@@ -56,6 +56,12 @@ class aaf_kv_stats(C.Structure):
     ]
 
 
+class aaf_kv_catalog_cols(C.Structure):
+    _fields_ = [("state_id", C.c_void_p), ("n_tokens", C.c_void_p), ("reuse", C.c_void_p), ("last_access", C.c_void_p),
+                ("block_offsets", C.c_void_p), ("block_id", C.c_void_p), ("pos_begin", C.c_void_p),
+                ("pos_end", C.c_void_p), ("refcount", C.c_void_p), ("address", C.c_void_p)]
+
+
 # every symbol include/aaf_kv.h declares: name -> (restype, argtypes)
 _vp, _i32, _i64, _u32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_size_t
 _p32 = C.POINTER(C.c_int32)
@@ -75,6 +81,8 @@ SYMBOLS = {
                                                   _i32, _p32, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host_chunked": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _i32, _p32, _vp]),
     "aaf_kv_evict_to_budget": (C.c_int, [_vp, C.c_double, C.c_double, C.c_double, _i64, _p32, _i32, _p32, _vp]),
+    "aaf_kv_catalog_rows": (C.c_int, [_vp, _p32, C.POINTER(_i64)]),
+    "aaf_kv_export_catalog": (C.c_int, [_vp, C.POINTER(aaf_kv_catalog_cols), _vp]),
     "aaf_kv_get_catalog": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
     "aaf_kv_ctx_len": (C.c_int, [_vp, _i32, C.POINTER(_i64)]),
     "aaf_kv_get_table": (C.c_int, [_vp, _i32, _p32, _i32, _p32]),
@@ -137,6 +145,8 @@ def aaf_kv_import_host_chunked(pool, src_host, desc, staging, staging_bytes, chu
     return _fn("aaf_kv_import_host_chunked")(pool, src_host, desc, staging, staging_bytes, chunk_tokens, out_ctx, stream)
 def aaf_kv_evict_to_budget(pool, alpha, beta, gamma, budget, out_victims, cap, n_victims, stream):
     return _fn("aaf_kv_evict_to_budget")(pool, alpha, beta, gamma, budget, out_victims, cap, n_victims, stream)
+def aaf_kv_catalog_rows(pool, n_states, n_rows): return _fn("aaf_kv_catalog_rows")(pool, n_states, n_rows)
+def aaf_kv_export_catalog(pool, cols, stream): return _fn("aaf_kv_export_catalog")(pool, cols, stream)
 def aaf_kv_get_catalog(pool, clock, reuse, last): return _fn("aaf_kv_get_catalog")(pool, clock, reuse, last)
 def aaf_kv_ctx_len(pool, ctx, out): return _fn("aaf_kv_ctx_len")(pool, ctx, out)
 def aaf_kv_get_table(pool, ctx, out, cap, n_blocks): return _fn("aaf_kv_get_table")(pool, ctx, out, cap, n_blocks)
@@ -302,6 +312,25 @@ class KVPool:
         if st != AAF_OK:
             raise RuntimeError(aaf_kv_strerror(st))
         return {"clock": clock.value, "reuse": reuse.tolist(), "last_access": last.tolist()}
+
+    def export_catalog(self) -> dict:
+        """Runs the columnar export into torch-allocated device buffers; returns the columns as torch tensors
+        (still on the device) trimmed to their row counts."""
+        torch = self.torch
+        ns, nr = C.c_int32(0), C.c_int64(0)
+        aaf_kv_catalog_rows(self.h, C.byref(ns), C.byref(nr))
+        i32 = lambda n: torch.empty(max(n, 1), dtype=torch.int32, device=self.device)
+        i64 = lambda n: torch.empty(max(n, 1), dtype=torch.int64, device=self.device)
+        t = {"state_id": i32(ns.value), "n_tokens": i64(ns.value), "reuse": i64(ns.value), "last_access": i64(ns.value),
+             "block_offsets": i32(ns.value + 1), "block_id": i32(nr.value), "pos_begin": i64(nr.value),
+             "pos_end": i64(nr.value), "refcount": i32(nr.value), "address": i64(nr.value)}
+        cols = aaf_kv_catalog_cols(**{k: v.data_ptr() for k, v in t.items()})
+        st = aaf_kv_export_catalog(self.h, C.byref(cols), self._stream())
+        if st != AAF_OK:
+            raise RuntimeError(aaf_kv_strerror(st))
+        n_of = lambda k: ns.value + 1 if k == "block_offsets" else (
+            ns.value if k in ("state_id", "n_tokens", "reuse", "last_access") else nr.value)
+        return {k: v[: n_of(k)] for k, v in t.items()}
 
     def materialize_host_chunked(self, ctx, t0, t1, dst_host, staging, chunk_tokens, flags=None):
         """flags: pinned torch int32 tensor receiving one completion flag per chunk (or None)."""

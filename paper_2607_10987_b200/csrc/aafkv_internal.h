@@ -117,4 +117,8 @@ cudaError_t launch_expire_wait(const DevState &s, long long limit_cycles, cudaSt
 cudaError_t launch_copy(int engine, const CopyTuning &t, const Geom &g, const DevState &s, int n_slots, int plane0,
                         int n_planes, long long avg_piece_bytes, int sm_count, cudaStream_t st);
 
+// columnar catalog export: state rows + offsets by a prefix scan (one CTA), block rows by a grid
+cudaError_t launch_export_catalog(const Geom &g, const DevState &s, const aaf_kv_catalog_cols &cols, int n_states,
+                                  long long n_block_rows, cudaStream_t st);
+
 }  // namespace aafkv

@@ -604,6 +604,56 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_to_budget_kernel(Geom g, D
 }
 
 // ------------------------------------------------------------------------------------------
+// columnar catalog export
+//   kernel 1 (one CTA): two exclusive prefix scans over the handles -- live flags give each state its
+//   row, block-table lengths give the list offsets -- and the state columns.
+//   kernel 2 (grid): one thread per block row; the row's state is found by binary search in the
+//   offsets, then the row is filled from the table and the reference counts (coalesced writes).
+__global__ void __launch_bounds__(PLAN_THREADS) export_states_kernel(Geom g, DevState s, aaf_kv_catalog_cols cols) {
+    int row_carry = 0, blk_carry = 0;
+    for (int base = 0; base < g.max_ctx; base += blockDim.x) {
+        const int c = base + threadIdx.x;
+        const long long len = c < g.max_ctx ? s.cat_len[c] : -1;
+        const int live = len >= 0;
+        const int nb = live ? (int)((len + g.BS - 1) / g.BS) : 0;
+        int live_tot, blk_tot;
+        const int row = row_carry + block_exclusive_scan(live, &live_tot);
+        const int off = blk_carry + block_exclusive_scan(nb, &blk_tot);
+        if (live) {
+            cols.state_id[row] = c;
+            cols.n_tokens[row] = len;
+            cols.reuse[row] = (long long)s.cat_reuse[c];
+            cols.last_access[row] = s.cat_last[c];
+            cols.block_offsets[row] = off;
+        }
+        row_carry += live_tot;
+        blk_carry += blk_tot;
+    }
+    if (threadIdx.x == 0) cols.block_offsets[row_carry] = blk_carry;
+}
+
+__global__ void __launch_bounds__(256) export_blocks_kernel(Geom g, DevState s, aaf_kv_catalog_cols cols,
+                                                            int n_states, long long n_rows) {
+    for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < n_rows;
+         r += (long long)gridDim.x * blockDim.x) {
+        int lo = 0, hi = n_states - 1;  // last state whose offset <= r
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (cols.block_offsets[mid] <= r) lo = mid; else hi = mid - 1;
+        }
+        const int c = cols.state_id[lo];
+        const long long j = r - cols.block_offsets[lo];
+        const long long len = cols.n_tokens[lo];
+        const int b = s.tables[(long long)c * g.max_blk + j];
+        cols.block_id[r] = b;
+        cols.pos_begin[r] = j * g.BS;
+        cols.pos_end[r] = min((j + 1) * g.BS, len);
+        cols.refcount[r] = s.refcount[b];
+        cols.address[r] = (long long)b * 2 * g.run;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // launchers
 
 static int grid_for(long long items, int threads, int cap) {
@@ -647,6 +697,15 @@ cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_export_catalog(const Geom &g, const DevState &s, const aaf_kv_catalog_cols &cols, int n_states,
+                                  long long n_block_rows, cudaStream_t st) {
+    export_states_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, cols);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || n_block_rows == 0) return e;
+    export_blocks_kernel<<<grid_for(n_block_rows, 256, 1184), 256, 0, st>>>(g, s, cols, n_states, n_block_rows);
     return cudaGetLastError();
 }
 

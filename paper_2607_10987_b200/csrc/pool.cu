@@ -772,6 +772,34 @@ int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gam
     return AAF_OK;
 }
 
+int aaf_kv_catalog_rows(aaf_kv_pool *p, int32_t *n_states, int64_t *n_block_rows) {
+    if (!p || !n_states || !n_block_rows) return AAF_ERR_INVALID_ARG;
+    long long rows = 0;
+    for (int c = 0; c < p->g.max_ctx; ++c)
+        if (p->len[c] >= 0) rows += nblk_of(p, p->len[c]);
+    *n_states = p->live_ctx;
+    *n_block_rows = rows;
+    return AAF_OK;
+}
+
+int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void *stream) {
+    if (!p || !cols) return AAF_ERR_INVALID_ARG;
+    int32_t ns = 0;
+    int64_t rows = 0;
+    aaf_kv_catalog_rows(p, &ns, &rows);
+    if (!cols->state_id || !cols->n_tokens || !cols->reuse || !cols->last_access || !cols->block_offsets)
+        return AAF_ERR_INVALID_ARG;
+    if (rows > 0 && (!cols->block_id || !cols->pos_begin || !cols->pos_end || !cols->refcount || !cols->address))
+        return AAF_ERR_INVALID_ARG;
+    if (rows > 0x7fffffffll) return AAF_ERR_TOO_LONG;  // Arrow int32 list offsets
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    if (launch_export_catalog(p->g, p->s, *cols, ns, rows, st) != cudaSuccess) return AAF_ERR_CUDA;
+    p->meta_launches += rows > 0 ? 2 : 1;
+    return AAF_OK;
+}
+
 int aaf_kv_get_catalog(aaf_kv_pool *p, int64_t *clock, int64_t *reuse_out, int64_t *last_access_out) {
     if (!p || !clock || !reuse_out || !last_access_out) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);

@@ -18,6 +18,15 @@ pytestmark = pytest.mark.gpu
 VEC, BULK, WARP = 1, 2, 3
 
 
+def same_catalog_export(gpu, cpu):
+    """columnar catalog export: every column identical to the oracle's"""
+    got = {k: v.cpu().numpy() for k, v in gpu.o.export_catalog().items()}
+    want = cpu.o.export_catalog()
+    assert got.keys() == want.keys()
+    for k in want:
+        assert got[k].dtype == want[k].dtype and np.array_equal(got[k], want[k]), k
+
+
 def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
     """Replays ops on the GPU library and on the oracle side by side and compares after every op."""
     layers = list(range(g.n_layers)) if layers is None else list(layers)
@@ -32,6 +41,7 @@ def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
             n = op["t1"] - op["t0"]
             assert np.array_equal(gpu.buf_layers(res_g, n, layers).reshape(-1), res_c), (i, op)
     assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view()), "pool image differs"
+    same_catalog_export(gpu, cpu)
     assert gpu.o.sync_status() == 0
     gs, cs = gpu.o.stats(), cpu.o.stats()
     for k in ("free_blocks", "live_blocks", "peak_live_blocks", "live_ctx", "cow_count"):
@@ -119,6 +129,7 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
         check_conservation(snap, g.n_blocks, g.block_size)
         if i % 8 == 7:
             assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view()), (i, kind)
+            same_catalog_export(gpu, cpu)
         outcomes.append((kind, st_c))
     assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view())
     assert gpu.o.sync_status() == 0
@@ -207,3 +218,27 @@ def test_scored_eviction_to_budget(weights, budget):
     assert gpu.o.evict_to_budget(float("nan"), 0.0, 1.0, 3)[0] == -1
     assert gpu.o.evict_to_budget(0.0, 0.0, 1.0, -2)[0] == -1
     assert gpu.o.sync_status() == 0
+
+
+def test_catalog_export_wraps_as_arrow_without_conversion():
+    import pyarrow as pa
+
+    g = Geometry(2, 2, 64, 4, 2, 64, 12, 32)
+    gpu = GpuBackend(g, 77)
+    cpu = OracleBackend(g, 77)
+    same_catalog_export(gpu, cpu)  # empty pool: no state rows, offsets = [0]
+    for be in (gpu, cpu):
+        a = be.imp(be.payload(77, 1, 10), 10)[1]
+        kids = be.fork(a, 3)[1]
+        be.append(kids[:2], [5, 1], [be.payload(77, 2, 5), be.payload(77, 3, 1)])
+        be.compose([kids[0], kids[2]], 0)
+        be.evict([kids[1]])
+    same_catalog_export(gpu, cpu)
+    cols = {k: v.cpu().numpy() for k, v in gpu.o.export_catalog().items()}
+    lst = pa.ListArray.from_arrays(pa.array(cols["block_offsets"], type=pa.int32()),
+                                   pa.array(cols["block_id"], type=pa.int32()))
+    lst.validate(full=True)
+    assert lst.to_pylist() == [gpu.o.table(int(c)).tolist() for c in cols["state_id"]]
+    tbl = pa.table({"state_id": cols["state_id"], "n_tokens": cols["n_tokens"], "reuse": cols["reuse"],
+                    "last_access": cols["last_access"], "blocks": lst})
+    assert tbl.num_rows == len(gpu.o.live_ctxs())
