@@ -48,7 +48,7 @@ struct DevState {
     DevCtl *ctl;
     int *refcount;   // [NB]
     int *ring;       // [NB]
-    int *last_pos;   // [NB] scratch of evict, -1 when idle
+    unsigned long long *last_pos;  // [NB] evict marks: (clock << 32) | last flattened position of the block
     int *tables;     // [max_ctx][max_blk]
     Piece *pieces;   // [max_pieces]
     int *scratch;    // [3 * max_batch] per-batch scratch of the append planner
@@ -99,7 +99,7 @@ cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEnt
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
                                 int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st);
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
-                         cudaStream_t st);
+                         long long clock, int *n_launches, cudaStream_t st);
 // Scored eviction (Alg. KV-Evict): result[0] = number of victims, result[1] = free blocks afterwards,
 // result[2..] = victims in eviction order; `result` is host memory the device can write.
 cudaError_t launch_evict_to_budget(const Geom &g, const DevState &s, double alpha, double beta, double gamma,

@@ -51,6 +51,14 @@ __device__ __forceinline__ void claim_block(const DevState &s, int b, int NB) {
     s.refcount[b] = 1;
 }
 
+// Adds a thread's byte count to the pool's payload counter: one atomic per warp instead of one per piece.
+// Must be called by all threads of the CTA (converged).
+__device__ __forceinline__ void add_payload(DevCtl *ctl, unsigned long long bytes) {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) bytes += __shfl_down_sync(0xffffffffu, bytes, d);
+    if ((threadIdx.x & 31) == 0 && bytes) atomicAdd(&ctl->payload_bytes, bytes);
+}
+
 // Argument records arrive in pinned host memory that the kernel reads over PCIe; every such read costs
 // a bus round trip and is not cached, so a kernel that searches its records stages them first: one
 // coalesced pass into shared memory (when they fit), then all further reads are on-chip.
@@ -248,6 +256,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 
     // phase 4: one thread per piece slot.  Slot piece_off[i] is entry i's copy-on-write piece, the
     // slots behind it are the blocks its new tokens touch, in table order.
+    unsigned long long my_bytes = 0;
     for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) {
         if (!ok) {
             s.pieces[sl].nbytes = 0;
@@ -277,7 +286,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
                 s.pieces[sl] = make_piece(pool_slot(g, old, 0), g.layer_stride, g.run, pool_slot(g, nb, 0),
                                           g.layer_stride, g.run, (unsigned)(r * g.row));
                 atomicAdd(&s.ctl->cow_count, 1ull);
-                atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(r * g.row * 2 * g.L));
+                my_bytes += (unsigned long long)(r * g.row * 2 * g.L);
             } else {
                 s.pieces[sl].nbytes = 0;
             }
@@ -296,8 +305,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
         s.pieces[sl] = make_piece(e.src + (tlo - T) * g.row, 2ll * e.n_new * g.row, (long long)e.n_new * g.row,
                                   pool_slot(g, b, tlo - jpos * g.BS), g.layer_stride, g.run,
                                   (unsigned)((thi - tlo) * g.row));
-        atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((thi - tlo) * g.row * 2 * g.L));
+        my_bytes += (unsigned long long)((thi - tlo) * g.row * 2 * g.L);
     }
+    add_payload(s.ctl, my_bytes);
     if (ok && s.cat_len)
         for (int i = threadIdx.x; i < n; i += blockDim.x) {
             s.cat_len[ent[i].ctx] = ent[i].T + ent[i].n_new;
@@ -334,6 +344,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
     if (!ok) {
         for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) s.pieces[sl].nbytes = 0;
     }
+    unsigned long long my_bytes = 0;
     for (int it = threadIdx.x; ok && it < total_work; it += blockDim.x) {
         int lo = 0, hi = m - 1;
         while (lo < hi) {
@@ -357,7 +368,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
                 s.pieces[sg.piece_off] = make_piece(pool_slot(g, st[full], 0), g.layer_stride, g.run,
                                                     pool_slot(g, nb, 0), g.layer_stride, g.run,
                                                     (unsigned)(rem * g.row));
-                atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(rem * g.row * 2 * g.L));
+                my_bytes += (unsigned long long)(rem * g.row * 2 * g.L);
             }
         } else {
             const long long nblk_off = (sg.off + g.BS - 1) / g.BS;
@@ -382,9 +393,10 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
             } else {
                 pp[1].nbytes = 0;
             }
-            atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((s_hi - s_lo) * g.row * 2 * g.L));
+            my_bytes += (unsigned long long)((s_hi - s_lo) * g.row * 2 * g.L);
         }
     }
+    add_payload(s.ctl, my_bytes);
     if (ok && s.cat_len)
         for (int i = threadIdx.x; i < m; i += blockDim.x) {  // every occurrence of a segment is one read
             atomicAdd(&s.cat_reuse[segs[i].ctx], 1ull);
@@ -408,58 +420,46 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
 
 // ------------------------------------------------------------------------------------------
 // evict
-//   kernel A (grid)  : every flattened entry drops one reference and records the largest
-//                      flattened position at which its block occurs in the batch.
-//   kernel B (1 CTA) : a block is freed by the entry at its LAST occurrence iff its count is now 0
-//                      (that is where the sequential loop would have freed it); freed ids are
-//                      compacted in flattened order by a prefix scan and pushed at the ring's tail.
-__device__ __forceinline__ int evict_entry_block(const Geom &g, const DevState &s, const int *ctx, const int *ent_off,
-                                                 int n, int e) {
-    int lo = 0, hi = n - 1;
+//   release : every flattened entry drops one reference and marks its block with
+//             stamp | position, keeping the largest (atomicMax): the block's LAST occurrence in the batch.
+//   push    : a block is freed by the entry at its last occurrence iff its count is now 0 (that is
+//             where the sequential loop would have freed it); freed ids are compacted in flattened
+//             order by a prefix scan and pushed at the ring's tail.
+//   The mark's high 32 bits are the call's logical clock, so marks of earlier calls are always
+//   smaller and the mark array never needs clearing.
+//   Small batches (<= EVICT_FUSED_MAX entries) run both phases in one CTA; larger ones run the release
+//   over a grid and the compaction in one CTA.
+constexpr int EVICT_STAGE = 2048;        // ints staged in shared memory: ctx[n] followed by ent_off[n + 1]
+constexpr int EVICT_ITEMS = 8;           // consecutive flattened entries per thread and pass
+constexpr int EVICT_FUSED_MAX = 32768;
+
+__device__ __forceinline__ int find_ctx_index(const int *ent_off, int n, int e) {
+    int lo = 0, hi = n - 1;  // last context whose first entry is <= e
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         if (ent_off[mid] <= e) lo = mid; else hi = mid - 1;
     }
-    return s.tables[(long long)ctx[lo] * g.max_blk + (e - ent_off[lo])];
+    return lo;
 }
 
-constexpr int EVICT_STAGE = 2048;  // ints: ctx[n] followed by ent_off[n + 1]
-
-__global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a,
-                                                            int n, int total) {
-    __shared__ int sh_args[EVICT_STAGE];
-    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
-    const int *ent_off = ctx + n;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
-        const int b = evict_entry_block(g, s, ctx, ent_off, n, e);
-        if (atomicSub(&s.refcount[b], 1) <= 0) set_status(s.ctl, AAF_ERR_CORRUPT, 7);
-        atomicMax(&s.last_pos[b], e);
-    }
+__device__ __forceinline__ void evict_release_entry(const Geom &g, const DevState &s, const int *ctx,
+                                                    const int *ent_off, int n, int e, unsigned long long stamp) {
+    const int ci = find_ctx_index(ent_off, n, e);
+    const int b = s.tables[(long long)ctx[ci] * g.max_blk + (e - ent_off[ci])];
+    if (atomicSub(&s.refcount[b], 1) <= 0) set_status(s.ctl, AAF_ERR_CORRUPT, 7);
+    atomicMax(&s.last_pos[b], stamp | (unsigned long long)(unsigned)e);
 }
 
-constexpr int EVICT_ITEMS = 8;  // consecutive flattened entries per thread and pass
-
-__global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
-                                                                  const EvictArgs *__restrict__ a, int n,
-                                                                  int total) {
-    __shared__ int sh_args[EVICT_STAGE];
-    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
-    const int *ent_off = ctx + n;
+// compaction of the freed blocks by one CTA (all threads of the CTA must call it)
+__device__ __forceinline__ void evict_push_phase(const Geom &g, const DevState &s, const int *ctx, const int *ent_off,
+                                                 int n, int total, unsigned long long stamp) {
     const unsigned long long tail0 = s.ctl->tail;
     int carry = 0;
     for (int base = 0; base < total; base += PLAN_THREADS * EVICT_ITEMS) {
         const int e0 = base + threadIdx.x * EVICT_ITEMS;
         int blk[EVICT_ITEMS];
         // locate the first entry once, then walk (context, position) forward: all table reads are independent
-        int ci = 0;
-        if (e0 < total) {
-            int lo = 0, hi = n - 1;
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (ent_off[mid] <= e0) lo = mid; else hi = mid - 1;
-            }
-            ci = lo;
-        }
+        int ci = e0 < total ? find_ctx_index(ent_off, n, e0) : 0;
 #pragma unroll
         for (int k = 0; k < EVICT_ITEMS; ++k) {
             const int e = e0 + k;
@@ -469,17 +469,18 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevSta
                 blk[k] = s.tables[(long long)ctx[ci] * g.max_blk + (e - ent_off[ci])];
             }
         }
-        int rc[EVICT_ITEMS], lp[EVICT_ITEMS];
+        int rc[EVICT_ITEMS];
+        unsigned long long lp[EVICT_ITEMS];
 #pragma unroll
         for (int k = 0; k < EVICT_ITEMS; ++k) {
             rc[k] = blk[k] >= 0 ? s.refcount[blk[k]] : 1;
-            lp[k] = blk[k] >= 0 ? s.last_pos[blk[k]] : -1;
+            lp[k] = blk[k] >= 0 ? s.last_pos[blk[k]] : 0ull;
         }
         int cnt = 0;
         unsigned flags = 0;
 #pragma unroll
         for (int k = 0; k < EVICT_ITEMS; ++k) {
-            const bool f = blk[k] >= 0 && rc[k] == 0 && lp[k] == e0 + k;
+            const bool f = blk[k] >= 0 && rc[k] == 0 && lp[k] == (stamp | (unsigned long long)(unsigned)(e0 + k));
             flags |= (f ? 1u : 0u) << k;
             cnt += f;
         }
@@ -493,16 +494,40 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevSta
             }
         carry += tot;
     }
-    __syncthreads();
-    // every flag has been taken: clear the scratch marks of the touched blocks
-    for (int e = threadIdx.x; e < total; e += blockDim.x)
-        s.last_pos[evict_entry_block(g, s, ctx, ent_off, n, e)] = -1;
     if (s.cat_len)
         for (int i = threadIdx.x; i < n; i += blockDim.x) s.cat_len[ctx[i]] = -1;
     if (threadIdx.x == 0) {
         if (tail0 + carry - s.ctl->head > (unsigned long long)g.NB) set_status(s.ctl, AAF_ERR_CORRUPT, 8);
         s.ctl->tail = tail0 + carry;
     }
+}
+
+__global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a,
+                                                            int n, int total, unsigned long long stamp) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    const int *ent_off = ctx + n;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x)
+        evict_release_entry(g, s, ctx, ent_off, n, e, stamp);
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
+                                                                  const EvictArgs *__restrict__ a, int n, int total,
+                                                                  unsigned long long stamp) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    evict_push_phase(g, s, ctx, ctx + n, n, total, stamp);
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) evict_fused_kernel(Geom g, DevState s,
+                                                                   const EvictArgs *__restrict__ a, int n, int total,
+                                                                   unsigned long long stamp) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    const int *ent_off = ctx + n;
+    for (int e = threadIdx.x; e < total; e += blockDim.x) evict_release_entry(g, s, ctx, ent_off, n, e, stamp);
+    __syncthreads();  // one CTA: every reference has been dropped and every mark set
+    evict_push_phase(g, s, ctx, ent_off, n, total, stamp);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -515,6 +540,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevSta
 __global__ void __launch_bounds__(PLAN_THREADS) evict_to_budget_kernel(Geom g, DevState s, double alpha, double beta,
                                                                        double gamma, long long budget,
                                                                        long long clock, int *result) {
+    const unsigned long long stamp = (unsigned long long)clock << 32;
     __shared__ double sh_score[32];
     __shared__ int sh_id[32];
     __shared__ int sh_victim;
@@ -566,10 +592,12 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_to_budget_kernel(Geom g, D
         // release the victim's entries
         const int nb = (int)((s.cat_len[v] + g.BS - 1) / g.BS);
         const int *table = s.tables + (long long)v * g.max_blk;
+        // marks grow from victim to victim (max_ctx * max_blk < 2^31), so none has to be cleared
+        const unsigned long long vstamp = stamp + (unsigned long long)nv * (unsigned long long)g.max_blk;
         for (int e = threadIdx.x; e < nb; e += blockDim.x) {
             const int b = table[e];
             if (atomicSub(&s.refcount[b], 1) <= 0) set_status(s.ctl, AAF_ERR_CORRUPT, 9);
-            atomicMax(&s.last_pos[b], e);
+            atomicMax(&s.last_pos[b], vstamp + (unsigned long long)(unsigned)e);
         }
         __syncthreads();
         const unsigned long long tail0 = s.ctl->tail;
@@ -579,15 +607,13 @@ __global__ void __launch_bounds__(PLAN_THREADS) evict_to_budget_kernel(Geom g, D
             int b = -1, flag = 0;
             if (e < nb) {
                 b = table[e];
-                flag = (s.refcount[b] == 0 && s.last_pos[b] == e);
+                flag = (s.refcount[b] == 0 && s.last_pos[b] == (vstamp + (unsigned long long)(unsigned)e));
             }
             int tot;
             const int ex = block_exclusive_scan(flag, &tot);
             if (flag) s.ring[(tail0 + (unsigned long long)(carry + ex)) % (unsigned long long)g.NB] = b;
             carry += tot;
         }
-        __syncthreads();
-        for (int e = threadIdx.x; e < nb; e += blockDim.x) s.last_pos[table[e]] = -1;
         if (threadIdx.x == 0) {
             s.ctl->tail = tail0 + carry;
             sh_live -= carry;
@@ -692,11 +718,18 @@ cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeS
     return cudaGetLastError();
 }
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
-                         cudaStream_t st) {
-    evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev, n, total);
+                         long long clock, int *n_launches, cudaStream_t st) {
+    const unsigned long long stamp = (unsigned long long)clock << 32;
+    if (total <= EVICT_FUSED_MAX) {
+        *n_launches = 1;
+        evict_fused_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp);
+        return cudaGetLastError();
+    }
+    *n_launches = 2;
+    evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev, n, total, stamp);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total);
+    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp);
     return cudaGetLastError();
 }
 

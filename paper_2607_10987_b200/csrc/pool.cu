@@ -5,7 +5,9 @@
 // guaranteed lower bound of the free-block count.  Block ids, reference counts and the ring live
 // on the device.  A call validates everything against the mirror, writes its argument records
 // into a pinned ring the planners read directly, and launches: planner kernel(s) then the copy
-// engine.  The device's free count is read back (one synchronising 16-byte copy) only when the
+// engine.  Planners run on a library-owned metadata stream and copies on the caller's stream, joined
+// by events and two alternating piece buffers, so the planner of the next operator runs while the
+// copy of the current one is still streaming.  The device's free count is read back (one synchronising 16-byte copy) only when the
 // lower bound cannot prove that a call fits, so out-of-blocks is reported exactly and
 // synchronously without a sync on the common path.
 #include <cuda_runtime.h>
@@ -50,9 +52,9 @@ Layout make_layout(const aaf_kv_pool_desc *d) {
     L.ctl = off; off = align_up(off + sizeof(DevCtl), 256);
     L.refcount = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
     L.ring = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
-    L.last_pos = off; off = align_up(off + sizeof(int) * (size_t)d->n_blocks, 256);
+    L.last_pos = off; off = align_up(off + sizeof(unsigned long long) * (size_t)d->n_blocks, 256);
     L.tables = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx * d->max_blocks_per_ctx, 256);
-    L.pieces = off; off = align_up(off + sizeof(Piece) * (size_t)L.max_pieces, 256);
+    L.pieces = off; off = align_up(off + 2 * sizeof(Piece) * (size_t)L.max_pieces, 256);  // two alternating buffers
     L.scratch = off; off = align_up(off + sizeof(int) * 3 * (size_t)L.max_batch, 256);
     L.cat_len = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
     L.cat_reuse = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
@@ -92,7 +94,13 @@ struct aaf_kv_pool {
     long long free_lb = 0;       // guaranteed lower bound of the device's free-block count
     long long clock = 0;         // logical clock: successful state-touching calls so far
     int *result = nullptr;       // pinned, device-writable: result of the scored eviction (max_ctx + 2 ints)
-    cudaStream_t last_stream = nullptr;
+    cudaStream_t last_stream = nullptr;  // the caller's stream of the most recent call (copies run there)
+    // Metadata kernels run on their own stream: they touch tables, reference counts, the ring and the piece
+    // buffers only, never payload, so the planner of operator i+1 can run while the copy of operator i is
+    // still streaming.  Two piece buffers alternate; events order planner -> copy and copy -> buffer reuse.
+    cudaStream_t meta_stream = nullptr;
+    cudaEvent_t plan_done[2] = {}, copy_done[2] = {};
+    int next_buf = 0;
     // pinned argument ring
     char *args = nullptr;
     size_t slot_bytes = 0;
@@ -142,8 +150,9 @@ void release_args(aaf_kv_pool *p, cudaStream_t st) {
 
 // exact free-block count: synchronises the stream and reads the ring counters
 int refresh_free(aaf_kv_pool *p, cudaStream_t st) {
+    (void)st;
     unsigned long long ht[2];
-    if (cudaStreamSynchronize(st) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess) return AAF_ERR_CUDA;  // the counters are metadata
     if (cudaMemcpy(ht, p->s.ctl, sizeof(ht), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
     p->free_lb = (long long)(ht[1] - ht[0]);
     return AAF_OK;
@@ -186,9 +195,36 @@ void drain_timing(aaf_kv_pool *p) {
 }
 
 // copy-engine launch for one operator class over planes [plane0, plane0 + n_planes)
-int run_copy(aaf_kv_pool *p, int cls, int n_slots, long long payload_tokens, cudaStream_t st, int piece0 = 0) {
+struct PlanSlot {
+    DevState view;  // device state whose `pieces` is the buffer this operator plans into
+    int buf;
+};
+
+// Before a planner: pick the next piece buffer and make the metadata stream wait until the copy launch
+// that last read that buffer has finished.
+PlanSlot begin_plan(aaf_kv_pool *p) {
+    PlanSlot ps;
+    ps.buf = p->next_buf;
+    ps.view = p->s;
+    ps.view.pieces = p->s.pieces + (size_t)ps.buf * (size_t)p->lay.max_pieces;
+    cudaStreamWaitEvent(p->meta_stream, p->copy_done[ps.buf], 0);
+    return ps;
+}
+// After the planner: the caller's stream (where the copy runs) waits for it.
+bool end_plan(aaf_kv_pool *p, const PlanSlot &ps, cudaStream_t st) {
+    return cudaEventRecord(p->plan_done[ps.buf], p->meta_stream) == cudaSuccess &&
+           cudaStreamWaitEvent(st, p->plan_done[ps.buf], 0) == cudaSuccess;
+}
+// After the operator's last copy launch: mark the buffer's readers done and switch buffers.
+void end_copy(aaf_kv_pool *p, const PlanSlot &ps, cudaStream_t st) {
+    cudaEventRecord(p->copy_done[ps.buf], st);
+    p->next_buf ^= 1;
+}
+
+int run_copy(aaf_kv_pool *p, const PlanSlot &ps, int cls, int n_slots, long long payload_tokens, cudaStream_t st,
+             int piece0 = 0) {
     const int plane0 = 0, n_planes = 2 * p->g.L;
-    DevState view = p->s;
+    DevState view = ps.view;
     view.pieces += piece0;  // a launch may cover a sub-range of the planned pieces (chunked transfers)
     const long long avg_piece = n_slots > 0 ? payload_tokens * p->g.row / n_slots : 0;
     if (n_slots <= 0) return AAF_OK;
@@ -230,13 +266,16 @@ int materialize_impl(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void
     const long long n = t1 - t0;
     if ((unsigned long long)dst_bytes < (unsigned long long)(n * bpt_of(p))) return AAF_ERR_DST_TOO_SMALL;
     p->last_stream = st;
-    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(dst_dev), p->clock + 1, st) !=
-        cudaSuccess)
+    const PlanSlot ps = begin_plan(p);
+    if (launch_plan_materialize(p->g, ps.view, ctx, t0, t1, static_cast<char *>(dst_dev), p->clock + 1,
+                                p->meta_stream) != cudaSuccess ||
+        !end_plan(p, ps, st))
         return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
     const int n_slots = (int)((t1 - 1) / p->g.BS - t0 / p->g.BS + 1);
-    const int rc = run_copy(p, AAF_OP_MATERIALIZE, n_slots, n, st);
+    const int rc = run_copy(p, ps, AAF_OP_MATERIALIZE, n_slots, n, st);
+    end_copy(p, ps, st);
     if (rc == AAF_OK && out_desc) fill_desc(p, out_desc, t0, n);
     return rc;
 }
@@ -259,7 +298,10 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
                             st) != cudaSuccess)
             return AAF_ERR_CUDA;
     }
-    if (launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(src_dev), p->clock + 1, st) != cudaSuccess)
+    const PlanSlot ps = begin_plan(p);
+    if (launch_plan_import(p->g, ps.view, c, n, static_cast<const char *>(src_dev), p->clock + 1, p->meta_stream) !=
+            cudaSuccess ||
+        !end_plan(p, ps, st))
         return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
@@ -267,7 +309,9 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
     p->len[c] = n;
     p->live_ctx += 1;
     *out_ctx = c;
-    return run_copy(p, AAF_OP_IMPORT, (int)nb, n, st);
+    const int rc = run_copy(p, ps, AAF_OP_IMPORT, (int)nb, n, st);
+    end_copy(p, ps, st);
+    return rc;
 }
 
 cudaEvent_t order_event(aaf_kv_pool *p) {
@@ -348,7 +392,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     p->s.ctl = reinterpret_cast<DevCtl *>(ws + lay.ctl);
     p->s.refcount = reinterpret_cast<int *>(ws + lay.refcount);
     p->s.ring = reinterpret_cast<int *>(ws + lay.ring);
-    p->s.last_pos = reinterpret_cast<int *>(ws + lay.last_pos);
+    p->s.last_pos = reinterpret_cast<unsigned long long *>(ws + lay.last_pos);
     p->s.tables = reinterpret_cast<int *>(ws + lay.tables);
     p->s.pieces = reinterpret_cast<Piece *>(ws + lay.pieces);
     p->s.scratch = reinterpret_cast<int *>(ws + lay.scratch);
@@ -366,6 +410,10 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
                    cudaSuccess;
     for (int i = 0; ok && i < ARG_SLOTS; ++i)
         ok = cudaEventCreateWithFlags(&p->slot_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&p->meta_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 2; ++i)
+        ok = cudaEventCreateWithFlags(&p->plan_done[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&p->copy_done[i], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc(reinterpret_cast<void **>(&p->result), sizeof(int) * ((size_t)desc->max_ctx + 2),
                              cudaHostAllocMapped) == cudaSuccess;
     // device state: counters, reference counts 0, ring, evict scratch -1
@@ -376,7 +424,6 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     ok = ok && cudaMemset(ws, 0, lay.tables) == cudaSuccess;
     ok = ok && cudaMemcpy(p->s.ctl, &ctl, sizeof(ctl), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(p->s.ring, ring.data(), sizeof(int) * ring.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemset(p->s.last_pos, 0xff, sizeof(int) * (size_t)desc->n_blocks) == cudaSuccess;
     ok = ok && cudaMemset(p->s.cat_len, 0xff, sizeof(long long) * (size_t)desc->max_ctx) == cudaSuccess;  // -1: free
     ok = ok && cudaMemset(p->s.cat_reuse, 0, lay.total - lay.cat_reuse) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -392,6 +439,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
 int aaf_kv_pool_destroy(aaf_kv_pool *p) {
     if (!p) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
+    if (p->meta_stream) cudaStreamSynchronize(p->meta_stream);
     if (p->last_stream || !p->pending.empty()) cudaStreamSynchronize(p->last_stream);
     for (auto &t : p->pending) {
         cudaEventDestroy(t.start);
@@ -403,6 +451,11 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
         cudaStreamDestroy(p->xfer_stream);
     }
     for (auto e : p->order_events) cudaEventDestroy(e);
+    for (int i = 0; i < 2; ++i) {
+        if (p->plan_done[i]) cudaEventDestroy(p->plan_done[i]);
+        if (p->copy_done[i]) cudaEventDestroy(p->copy_done[i]);
+    }
+    if (p->meta_stream) cudaStreamDestroy(p->meta_stream);
     for (int i = 0; i < ARG_SLOTS; ++i)
         if (p->slot_ev[i]) cudaEventDestroy(p->slot_ev[i]);
     if (p->args) cudaFreeHost(p->args);
@@ -473,8 +526,10 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     p->last_stream = st;
     if (done_flags_host)
         for (int c = 0; c < n_chunks; ++c) done_flags_host[c] = 0;
-    if (launch_plan_materialize(p->g, p->s, ctx, t0, t1, static_cast<char *>(staging_dev), p->clock + 1, st) !=
-        cudaSuccess)
+    const PlanSlot ps = begin_plan(p);
+    if (launch_plan_materialize(p->g, ps.view, ctx, t0, t1, static_cast<char *>(staging_dev), p->clock + 1,
+                                p->meta_stream) != cudaSuccess ||
+        !end_plan(p, ps, st))
         return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
@@ -482,7 +537,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     for (int c = 0; c < n_chunks && ok; ++c) {
         const int s0 = c * per_chunk, s1 = std::min(n_slots, s0 + per_chunk);
         const long long lo = std::max<long long>(t0, (j0 + s0) * BS), hi = std::min<long long>(t1, (j0 + s1) * BS);
-        ok = run_copy(p, AAF_OP_MATERIALIZE, s1 - s0, hi - lo, st, s0) == AAF_OK;  // gather of this chunk's blocks
+        ok = run_copy(p, ps, AAF_OP_MATERIALIZE, s1 - s0, hi - lo, st, s0) == AAF_OK;  // gather of this chunk's blocks
         cudaEvent_t ev = order_event(p);
         ok = ok && ev && cudaEventRecord(ev, st) == cudaSuccess &&
              cudaStreamWaitEvent(p->xfer_stream, ev, 0) == cudaSuccess;
@@ -493,6 +548,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
             ok = cudaMemcpyAsync(&done_flags_host[c], &p->s.ctl->one, sizeof(uint32_t), cudaMemcpyDeviceToHost,
                                  p->xfer_stream) == cudaSuccess;
     }
+    end_copy(p, ps, st);
     // the caller's stream is complete only when the last chunk has landed
     cudaEvent_t fin = order_event(p);
     ok = ok && fin && cudaEventRecord(fin, p->xfer_stream) == cudaSuccess && cudaStreamWaitEvent(st, fin, 0) == cudaSuccess;
@@ -526,8 +582,10 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     cudaEvent_t start = order_event(p);
     bool ok = start && cudaEventRecord(start, st) == cudaSuccess &&
               cudaStreamWaitEvent(p->xfer_stream, start, 0) == cudaSuccess;
-    ok = ok && launch_plan_import(p->g, p->s, c, n, static_cast<const char *>(staging_dev), p->clock + 1, st) ==
-                   cudaSuccess;
+    const PlanSlot ps = begin_plan(p);
+    ok = ok && launch_plan_import(p->g, ps.view, c, n, static_cast<const char *>(staging_dev), p->clock + 1,
+                                  p->meta_stream) == cudaSuccess &&
+         end_plan(p, ps, st);
     if (!ok) return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
@@ -545,8 +603,9 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
         ok = ok && ev && cudaEventRecord(ev, p->xfer_stream) == cudaSuccess &&
              cudaStreamWaitEvent(st, ev, 0) == cudaSuccess;
         // scatter of the chunk that has arrived, while the next one crosses PCIe
-        ok = ok && run_copy(p, AAF_OP_IMPORT, (int)(s1 - s0), hi - lo, st, (int)s0) == AAF_OK;
+        ok = ok && run_copy(p, ps, AAF_OP_IMPORT, (int)(s1 - s0), hi - lo, st, (int)s0) == AAF_OK;
     }
+    end_copy(p, ps, st);
     return ok ? AAF_OK : AAF_ERR_CUDA;
 }
 
@@ -565,8 +624,8 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
         children[j] = c;
     }
     const long long T = p->len[parent];
-    const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, children, p->clock + 1, st);
-    release_args(p, st);
+    const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, children, p->clock + 1, p->meta_stream);
+    release_args(p, p->meta_stream);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
@@ -624,8 +683,9 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             // the worst case does not fit: ask the planner (dry run) how many blocks the batch really
             // needs; only tail blocks that are still shared are copied
             unsigned long long need = 0;
-            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, p->clock, st) != cudaSuccess ||
-                cudaStreamSynchronize(st) != cudaSuccess ||
+            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, p->clock, p->meta_stream) !=
+                    cudaSuccess ||
+                cudaStreamSynchronize(p->meta_stream) != cudaSuccess ||
                 cudaMemcpy(&need, &p->s.ctl->probe_need, sizeof(need), cudaMemcpyDeviceToHost) != cudaSuccess)
                 rc = AAF_ERR_CUDA;
             else if ((long long)need > p->free_lb)
@@ -634,19 +694,22 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             charge = (long long)need;
         }
         if (rc != AAF_OK) {
-            release_args(p, st);
+            release_args(p, p->meta_stream);
             return rc;
         }
     }
-    const cudaError_t e =
-        launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 0, p->clock + 1, st);
-    release_args(p, st);
-    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    const PlanSlot ps = begin_plan(p);
+    const cudaError_t e = launch_plan_append(p->g, ps.view, ent, n, (int)slots, p->lay.max_batch, 0, p->clock + 1,
+                                             p->meta_stream);
+    release_args(p, p->meta_stream);
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= charge;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] += n_new[i];
-    return run_copy(p, AAF_OP_APPEND, (int)slots, append_tokens, st);
+    const int rc_copy = run_copy(p, ps, AAF_OP_APPEND, (int)slots, append_tokens, st);
+    end_copy(p, ps, st);
+    return rc_copy;
 }
 
 int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
@@ -695,17 +758,20 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     p->last_stream = st;
     ComposeSeg *dev_rec = reinterpret_cast<ComposeSeg *>(acquire_args(p));
     memcpy(dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
-    const cudaError_t e =
-        launch_plan_compose(p->g, p->s, dev_rec, m, (int)work, (int)fresh, (int)slots, c, p->clock + 1, st);
-    release_args(p, st);
-    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    const PlanSlot ps = begin_plan(p);
+    const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, m, (int)work, (int)fresh, (int)slots, c,
+                                              p->clock + 1, p->meta_stream);
+    release_args(p, p->meta_stream);
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return AAF_ERR_CUDA;
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= fresh;
     p->len[c] = off;
     p->live_ctx += 1;
     *out_ctx = c;
-    return run_copy(p, AAF_OP_COMPOSE, (int)slots, copied_tokens, st);
+    const int rc_copy = run_copy(p, ps, AAF_OP_COMPOSE, (int)slots, copied_tokens, st);
+    end_copy(p, ps, st);
+    return rc_copy;
 }
 
 int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {
@@ -733,11 +799,12 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
     ent_off[n] = (int)total;
     a->n = n;
     a->total = (int)total;
-    const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, st);
-    release_args(p, st);
+    int n_launches = 0;
+    const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, p->clock + 1, &n_launches, p->meta_stream);
+    release_args(p, p->meta_stream);
     if (e != cudaSuccess) return AAF_ERR_CUDA;
     p->clock += 1;
-    p->meta_launches += 2;
+    p->meta_launches += n_launches;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] = -1;
     p->live_ctx -= n;
     return AAF_OK;  // the lower bound of the free count stays valid: evict only adds free blocks
@@ -753,12 +820,12 @@ int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gam
     DeviceGuard guard(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
-    if (launch_evict_to_budget(p->g, p->s, alpha, beta, gamma, budget_blocks, p->clock + 1, p->result, st) !=
-        cudaSuccess)
+    if (launch_evict_to_budget(p->g, p->s, alpha, beta, gamma, budget_blocks, p->clock + 1, p->result,
+                               p->meta_stream) != cudaSuccess)
         return AAF_ERR_CUDA;
     p->meta_launches += 1;
     // the victims are chosen on the device; the host mirror needs them before the next call
-    if (cudaStreamSynchronize(st) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess) return AAF_ERR_CUDA;
     p->clock += 1;
     const int nv = p->result[0];
     for (int i = 0; i < nv; ++i) {
@@ -795,7 +862,11 @@ int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void 
     DeviceGuard guard(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
-    if (launch_export_catalog(p->g, p->s, *cols, ns, rows, st) != cudaSuccess) return AAF_ERR_CUDA;
+    // the columns are the caller's buffers: written on the metadata stream, then the caller's stream waits
+    cudaEvent_t done = order_event(p);
+    if (launch_export_catalog(p->g, p->s, *cols, ns, rows, p->meta_stream) != cudaSuccess || !done ||
+        cudaEventRecord(done, p->meta_stream) != cudaSuccess || cudaStreamWaitEvent(st, done, 0) != cudaSuccess)
+        return AAF_ERR_CUDA;
     p->meta_launches += rows > 0 ? 2 : 1;
     return AAF_OK;
 }
@@ -803,7 +874,8 @@ int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void 
 int aaf_kv_get_catalog(aaf_kv_pool *p, int64_t *clock, int64_t *reuse_out, int64_t *last_access_out) {
     if (!p || !clock || !reuse_out || !last_access_out) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     const size_t nbytes = sizeof(long long) * (size_t)p->g.max_ctx;
     if (cudaMemcpy(reuse_out, p->s.cat_reuse, nbytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
         cudaMemcpy(last_access_out, p->s.cat_last, nbytes, cudaMemcpyDeviceToHost) != cudaSuccess)
@@ -827,7 +899,8 @@ int aaf_kv_get_table(aaf_kv_pool *p, aaf_ctx_t ctx, int32_t *host_out, int32_t c
     const long long nb = nblk_of(p, p->len[ctx]);
     if (cap < nb) return AAF_ERR_DST_TOO_SMALL;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     if (cudaMemcpy(host_out, p->s.tables + (long long)ctx * p->g.max_blk, sizeof(int) * (size_t)nb,
                    cudaMemcpyDeviceToHost) != cudaSuccess)
         return AAF_ERR_CUDA;
@@ -838,7 +911,8 @@ int aaf_kv_get_table(aaf_kv_pool *p, aaf_ctx_t ctx, int32_t *host_out, int32_t c
 int aaf_kv_get_refcounts(aaf_kv_pool *p, int32_t *host_out) {
     if (!p || !host_out) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     return cudaMemcpy(host_out, p->s.refcount, sizeof(int) * (size_t)p->g.NB, cudaMemcpyDeviceToHost) == cudaSuccess
                ? AAF_OK
                : AAF_ERR_CUDA;
@@ -847,7 +921,8 @@ int aaf_kv_get_refcounts(aaf_kv_pool *p, int32_t *host_out) {
 int aaf_kv_get_free_list(aaf_kv_pool *p, int32_t *host_out, int32_t *n_free) {
     if (!p || !host_out || !n_free) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     unsigned long long ht[2];
     std::vector<int> ring((size_t)p->g.NB);
     if (cudaMemcpy(ht, p->s.ctl, sizeof(ht), cudaMemcpyDeviceToHost) != cudaSuccess ||
@@ -864,7 +939,8 @@ int aaf_kv_get_free_list(aaf_kv_pool *p, int32_t *host_out, int32_t *n_free) {
 int aaf_kv_pool_stats(aaf_kv_pool *p, aaf_kv_stats *out) {
     if (!p || !out) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     drain_timing(p);
     DevCtl ctl;
     if (cudaMemcpy(&ctl, p->s.ctl, sizeof(ctl), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
@@ -888,7 +964,8 @@ int aaf_kv_pool_stats(aaf_kv_pool *p, aaf_kv_stats *out) {
 int aaf_kv_sync_status(aaf_kv_pool *p) {
     if (!p) return AAF_ERR_INVALID_ARG;
     DeviceGuard guard(p->device);
-    if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess || cudaStreamSynchronize(p->last_stream) != cudaSuccess)
+        return AAF_ERR_CUDA;
     int st[2] = {0, 0};
     if (cudaMemcpy(st, &p->s.ctl->status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return AAF_ERR_CUDA;
     if (st[0] != 0) {
@@ -910,7 +987,7 @@ int aaf_kv_debug_expire_wait(aaf_kv_pool *p, uint64_t limit_cycles, void *stream
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
     p->meta_launches += 1;
-    return launch_expire_wait(p->s, (long long)limit_cycles, st) == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
+    return launch_expire_wait(p->s, (long long)limit_cycles, p->meta_stream) == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
 }
 
 int aaf_kv_set_timing(aaf_kv_pool *p, int enable) {
