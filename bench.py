@@ -104,7 +104,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -397,7 +397,7 @@ def extra_report(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer"])
@@ -423,10 +423,15 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    dev_index = local_rank % torch.cuda.device_count()  # one rank per GPU; the modulo only matters in self-tests
+    torch.cuda.set_device(dev_index)
+    dev = torch.device("cuda", dev_index)
+    backend = os.environ.get("AAFKV_BENCH_DIST_BACKEND", "nccl")  # control plane only: barrier + max of the time
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
 
     g, seed, T, agents, n_new = w["g"], w["seed"], w["T"], w["agents"], w["n_new"]
     free_b, _total = torch.cuda.mem_get_info(dev)
@@ -435,7 +440,7 @@ def main():
     while need(n_blocks) > free_b and n_blocks > 4096:
         n_blocks //= 2  # recorded in config.n_blocks when the device lacks memory for the full pool
     pool = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, n_blocks, g.max_ctx,
-                  g.max_blocks_per_ctx, free_order=configs.free_order(seed, n_blocks), device=local_rank)
+                  g.max_blocks_per_ctx, free_order=configs.free_order(seed, n_blocks), device=dev_index)
     pool.set_copy_engine(args.engine)
     elems = lambda n: g.n_layers * 2 * n * g.row // 2
     root_buf = fill.fill_torch(seed, 1, 0, elems(T), dev).view(torch.uint8)
@@ -459,7 +464,7 @@ def main():
         barrier()
         ms = e0.elapsed_time(e1)
         if world > 1:
-            t = torch.tensor([ms], device=dev)
+            t = torch.tensor([ms], device=dev if backend == "nccl" else "cpu")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             ms = float(t.item())
         return ms
@@ -471,7 +476,7 @@ def main():
     s0 = pool.stats()
     pool.set_timing(True)
     vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
-    smi_id = vis.split(",")[local_rank].strip() if vis and local_rank < len(vis.split(",")) else str(local_rank)
+    smi_id = vis.split(",")[dev_index].strip() if vis and dev_index < len(vis.split(",")) else str(dev_index)
     sampler = ClockSampler(smi_id) if rank == 0 else None
     ms = run(args.steps, dev_step)
     clocks = sampler.stop() if sampler else None
