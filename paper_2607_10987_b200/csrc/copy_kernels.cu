@@ -1,17 +1,20 @@
-// Copy engines of libaafkv.so: every byte a KV operator moves goes through one of the two
-// kernels below.  Both consume the same piece list (see Piece): a launch covers
+// Copy engines of libaafkv.so: every byte a KV operator moves goes through one of the three
+// kernels below.  All consume the same piece list (see Piece): a launch covers
 // n_slots pieces x n_planes (layer, K/V) planes, split into chunks of at most `chunk` bytes.
 //
 // The path is pure streaming (each byte is read once and written once, nothing is reused), so
 // the bound is HBM bandwidth: what matters is enough independent 16-byte accesses in flight per
-// SM, fully coalesced, and a grid that is a multiple of the SM count.
+// SM, fully coalesced, and a persistent grid of exactly one resident wave (a multiple of the SM count).
 //
-//   VEC  : 256 threads per CTA, each thread keeps UNROLL 16-byte streaming loads in flight and
-//          then stores them; grid-stride over chunks with a persistent grid.
 //   BULK : one elected thread per CTA drives a ring of shared-memory stages with
 //          cp.async.bulk (global -> shared, completion on an mbarrier) and
-//          cp.async.bulk (shared -> global, bulk async-group); no registers touch the data.
-//          Every wait is bounded; on expiry the kernel records AAF_ERR_TIMEOUT and leaves.
+//          cp.async.bulk (shared -> global, bulk async-group); no registers touch the data and the
+//          SMs stay idle.  Every wait is bounded; on expiry the kernel records AAF_ERR_TIMEOUT and
+//          leaves.  The default for pieces of about a run.
+//   WARP : 16-byte streaming loads/stores scheduled per warp, 32 units decoded at once; the default
+//          for small and ragged pieces.
+//   VEC  : 256 threads per CTA, each thread keeps UNROLL 16-byte streaming loads in flight and
+//          then stores them; one chunk per CTA iteration.  Kept as the plain baseline.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -21,7 +24,7 @@
 namespace aafkv {
 
 // ------------------------------------------------------------------------------------------
-// unit decomposition shared by both engines: unit u -> (chunk c, piece p, plane q), plane-major
+// unit decomposition shared by all engines: unit u -> (chunk c, piece p, plane q), plane-major
 // so that neighbouring CTAs stream neighbouring addresses of the dense side.
 struct Unit {
     const char *src;
