@@ -242,3 +242,52 @@ def test_catalog_export_wraps_as_arrow_without_conversion():
     tbl = pa.table({"state_id": cols["state_id"], "n_tokens": cols["n_tokens"], "reuse": cols["reuse"],
                     "last_access": cols["last_access"], "blocks": lst})
     assert tbl.num_rows == len(gpu.o.live_ctxs())
+
+
+# degenerate and extreme geometries: one-token blocks, 16-byte rows, odd block sizes, a single handle,
+# runs larger than every engine's chunk
+EDGE_GEOMETRIES = [
+    Geometry(1, 1, 8, 1, 2, 40, 6, 24),        # block = 1 token, row = 16 B, run = 16 B
+    Geometry(2, 1, 8, 3, 2, 50, 5, 20),        # row 16 B, block of 3 tokens
+    Geometry(1, 8, 128, 64, 2, 24, 4, 8),      # run = 128 KiB (> bulk chunk, several chunks per piece)
+    Geometry(5, 2, 24, 5, 4, 64, 7, 16),       # 4-byte elements, row 192 B, run 960 B
+    Geometry(1, 1, 8, 4, 2, 12, 1, 12),        # a single context handle
+]
+
+
+@pytest.mark.parametrize("engine", [0, VEC, BULK, WARP])
+@pytest.mark.parametrize("gi", range(len(EDGE_GEOMETRIES)))
+def test_random_walks_on_edge_geometries(engine, gi):
+    g = EDGE_GEOMETRIES[gi]
+    outcomes = random_walk(g, 8100 + gi, 120, engine)
+    assert sum(st == 0 for _, st in outcomes) >= 25
+
+
+def test_capacity_limits_are_exact():
+    """Longest table, largest batch, last free block, last free handle: accepted at the limit, refused one past it."""
+    g = Geometry(1, 1, 8, 2, 2, 64, 6, 10)
+    gpu = GpuBackend(g, 3, max_batch=4)
+    cpu = OracleBackend(g, 3)
+    for be in (gpu, cpu):
+        pay = lambda s, n: be.payload(3, s, n)
+        assert be.imp(pay(1, 20), 20) == (0, 0)                                   # exactly max_blocks_per_ctx blocks
+        assert be.imp(pay(2, 21), 21)[0] == -5                                    # one token too long
+        assert be.append([0], [1], [pay(3, 1)])[0] == -5
+        assert be.fork(0, 4) == (0, [1, 2, 3, 4])                                 # k = max_batch
+        assert be.compose([1, 2], 0)[0] == -5                                     # 40 tokens > 10 blocks
+        assert be.evict([1, 2, 3, 4])[0] == 0                                     # n = max_batch
+        assert be.imp(pay(4, 19), 19) == (0, 1)                                   # 10 more blocks
+        assert be.fork(1, 4) == (0, [2, 3, 4, 5])                                 # uses the last free handle
+        assert be.imp(pay(5, 1), 1)[0] == -4                                      # no handle left
+        assert be.evict([5])[0] == 0
+        assert be.append([1, 2, 3, 4], [1, 1, 1, 1], [pay(6 + i, 1) for i in range(4)])[0] == 0  # 3 COW + in place
+    assert gpu.o.fork(0, 5)[0] == binding_too_many()
+    assert gpu.snapshot() == cpu.snapshot()
+    assert np.array_equal(gpu.pool_layers([0]), cpu.o.pool_view())
+    assert gpu.o.stats()["cow_count"] == cpu.o.stats()["cow_count"] == 3
+
+
+def binding_too_many():
+    from paper_2607_10987_b200 import binding
+
+    return binding.AAF_ERR_TOO_MANY
