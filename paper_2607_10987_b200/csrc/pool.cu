@@ -40,7 +40,7 @@ bool geometry_ok(const aaf_kv_pool_desc *d) {
     const long long row = (long long)d->n_kv_heads * d->head_dim * d->elt_bytes;
     if (row % 16 != 0) return false;
     if (row * d->block_size > (1ll << 30)) return false;  // a run must fit the 32-bit piece size
-    if ((long long)d->max_ctx * d->max_blocks_per_ctx > (1ll << 31)) return false;
+    if ((long long)d->max_ctx * d->max_blocks_per_ctx >= (1ll << 31)) return false;  // flattened entry indices are ints
     return true;
 }
 
