@@ -34,7 +34,12 @@
  * library allocates host memory only (the pool object, a pinned argument ring, events).
  *
  * Ordering: calls on one pool are applied in call order and must be issued to one stream
- * (or the caller orders streams itself).  Data calls are asynchronous.  Not thread-safe
+ * (or the caller orders streams itself).  Data calls are asynchronous.  Every kernel that
+ * touches payload bytes (pool rows, transfer buffers) runs on the `stream` argument, so the
+ * caller's own work on that stream is ordered against them as usual.  Kernels that touch only
+ * the library's metadata (block tables, reference counts, the ring, copy descriptors) run on a
+ * library-owned stream that the library orders against `stream` with events; metadata is
+ * visible only through the introspection calls, which synchronise both.  Not thread-safe
  * per pool.  Pointers marked (device) must be device pointers, 16-byte aligned; row must
  * be a multiple of 16.  Pointers marked (host) are ordinary host pointers read or
  * written before the call returns.

@@ -101,3 +101,51 @@ def test_scaled_trace_8b_rows(bs, n_ops):
     nb = int(0.75 * demand)
     d, stats = lockstep_churn(make(nb), cap, n_ops, snap_every=100, pool_every=500, buf_every=3, **kw)
     assert any(st == churn.OOM_BLOCKS for _, _, st in d.log)
+
+
+def test_full_size_trace_8b_pool_metadata_against_small_row_oracle():
+    """The trace exactly as the benchmark runs it (8B rows, 32 layers, pool = 75 % of demand, about 60 GiB)
+    on the GPU, against the oracle run with 16-byte rows: tables, reference counts, free list, catalog and
+    every status depend on token counts only, so they must agree call by call although the rows differ.
+    Bytes at this size are covered by a property that holds at any size: a transfer round trip
+    reproduces its source (materialize(import(materialize(c))) == materialize(c)), checked on the GPU."""
+    import torch
+
+    bs, cap = 16, 32768
+    small = lambda nb: Geometry(1, 1, 8, bs, 2, nb, 80, cap // bs)
+    demand = demand_blocks(small, cap, bs, 10000)
+    nb = int(0.75 * demand)
+    g = Geometry(32, 8, 128, bs, 2, nb, 80, cap // bs)
+    free_b, _ = torch.cuda.mem_get_info()
+    if g.pool_bytes + (14 << 30) > free_b:
+        pytest.skip("not enough free device memory for the benchmark-sized pool")
+    order = configs.free_order(SEED, nb)
+    gpu = GpuBackend(g, SEED, free_order=order, init_fill=False, staging_tokens=cap)
+    cpu = OracleBackend(small(nb), SEED, free_order=order, init_fill=False)
+    dg = churn.ChurnDriver(gpu, SEED, max_ctx_tokens=cap)
+    dc = churn.ChurnDriver(cpu, SEED, max_ctx_tokens=cap)
+    second = torch.empty(cap * g.bpt, dtype=torch.uint8, device=gpu.o.device)
+    checked = 0
+    for i in range(10000):
+        k = len(dc.log)
+        dc.step()
+        dg.step()
+        assert dg.log[k:] == dc.log[k:], (i, dg.log[k:], dc.log[k:])
+        new = dc.log[k:]
+        if len(new) >= 2 and new[-2][0] == "materialize" and new[-1] == ("import", (new[-2][1][2],), 0) and i % 40 == 0:
+            # round trip just happened: staging still holds materialize(src); the newest context is its import
+            n = new[-2][1][2]
+            newest = [s for s in dg.slots if s is not None and s[2] == dg.clock and s[1] == n][-1][0]
+            st, again = gpu.o.materialize(newest, 0, n, out=second[: n * g.bpt])
+            assert st == 0 and torch.equal(again, gpu.staging[: n * g.bpt]), i
+            assert cpu.o.materialize(newest, 0, n)[0] == 0  # the same extra read on the oracle keeps the clocks equal
+            checked += 1
+        if (i + 1) % 1000 == 0:
+            assert gpu.snapshot() == cpu.snapshot(), i
+            assert gpu.o.catalog() == cpu.o.catalog(), i
+    assert checked >= 5
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+    gs, cs = gpu.o.stats(), cpu.o.stats()
+    for key in ("free_blocks", "peak_live_blocks", "cow_count", "live_ctx"):
+        assert gs[key] == cs[key]
+    assert gs["payload_bytes"] == cs["rows_copied"] * g.row * g.n_layers  # same rows moved, full-size bytes
