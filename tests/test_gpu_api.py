@@ -181,3 +181,39 @@ def test_chunked_host_transfer_is_byte_identical_and_flags_every_chunk(chunk_tok
     assert gpu.o.materialize_host_chunked(c, t0, t1, h_dst, staging, 16, flags[:3])[0] == binding.AAF_ERR_DST_TOO_SMALL
     assert gpu.o.import_host_chunked(h_src, n, staging, 0)[0] == binding.AAF_ERR_INVALID_ARG
     assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+
+
+def test_two_pools_of_different_geometry_interleaved():
+    """Launch shapes and scratch are per pool: two pools with different rows, block sizes and engines,
+    used alternately on the same stream, each stay bit-exact against their own oracle."""
+    ga = Geometry(2, 8, 128, 16, 2, 128, 8, 64)   # 2 KiB rows, 32 KiB runs
+    gb = Geometry(3, 1, 8, 5, 2, 160, 8, 64)      # 16-byte rows, 80-byte runs
+    pairs = []
+    for g, seed, engine in ((ga, 11, 0), (gb, 12, 0)):
+        order = configs.free_order(seed, g.n_blocks)
+        pairs.append((g, seed, GpuBackend(g, seed, free_order=order, engine=engine),
+                      OracleBackend(g, seed, free_order=order)))
+    script = [("imp", 70), ("fork", 2), ("append", 9), ("compose", None), ("mat", None), ("evict", None), ("imp", 33)]
+    for step, arg in script:
+        for g, seed, gpu, cpu in pairs:  # alternate pools at every operator
+            for be in (gpu, cpu):
+                if step == "imp":
+                    assert be.imp(be.payload(seed, 1 + arg, arg), arg)[0] == 0
+                elif step == "fork":
+                    assert be.fork(0, arg)[0] == 0
+                elif step == "append":
+                    assert be.append([1, 2], [arg, arg + 1], [be.payload(seed, 5, arg), be.payload(seed, 6, arg + 1)])[0] == 0
+                elif step == "compose":
+                    assert be.compose([1, 0, 2], 0)[0] == 0
+                elif step == "evict":
+                    assert be.evict([0, 2])[0] == 0
+            if step == "mat":
+                n = cpu.o.ctx_len(3)
+                sg, bg = gpu.materialize(3, 0, n)
+                sc, bc = cpu.materialize(3, 0, n)
+                assert sg == sc == 0
+                assert np.array_equal(gpu.buf_layers(bg, n, range(g.n_layers)).reshape(-1), bc)
+    for g, seed, gpu, cpu in pairs:
+        assert gpu.snapshot() == cpu.snapshot()
+        assert np.array_equal(gpu.pool_layers(range(g.n_layers)), cpu.o.pool_view())
+        assert gpu.o.sync_status() == 0

@@ -1,10 +1,10 @@
 """Churn workload: a seeded stream of agent operations under memory pressure (harness code).
 
 64 agent slots; 10,000 operations drawn with the mix 30 % append, 20 % fork, 20 % compose,
-15 % transfer round trip (materialize + import), 15 % evict; segment lengths lognormal with median
-2048 tokens.  The pool is capped at 75 % of the demand (= peak live blocks of the same seed on an
-unbounded pool), and the caller's eviction policy is LRU: when an operator reports out-of-blocks
-the driver evicts the least recently used agent that the operator does not use and retries.  That
+15 % transfer (materialize / import), 15 % evict; segment lengths lognormal with median 2048 tokens.
+The pool is capped at 75 % of the demand (= peak live blocks of the same seed on a pool that never
+runs out), and the caller's eviction policy is LRU: when an operator reports out-of-blocks the
+driver evicts the least recently used agent that the operator does not use and retries.  That
 policy is the caller's side of Alg. "KV-Evict" (score = -age); the library only releases blocks.
 
 The driver knows nothing about blocks: it tracks handles, token counts and LRU stamps, calls the
@@ -16,11 +16,17 @@ Payloads: every import/append reads a window of one pre-generated stream (worklo
 1), so that generating inputs costs nothing per operation.  ``backend.window(op_index, n_tokens)``
 returns the n-token transfer buffer that starts at element ``(op_index * 8) % slack`` of it.
 
-Details the workload description leaves open and this driver fixes: lengths = round(lognormal(
-mu = ln 2048, sigma = 0.8)) clamped to [1, 16384]; contexts capped at 65536 tokens (appends are
-shortened, trailing compose segments dropped); fork fan-out k in {1, 2, 4, 8}; compose arity in
-{2, 3, 4} over distinct live agents; new contexts go to the lowest empty slot, else they replace the
-least recently used slot the operator does not use.
+Details the workload description leaves open and this driver fixes:
+  * lengths = round(lognormal(mu = ln median, sigma = 0.8)) clamped to [1, max_seg_tokens];
+  * contexts are capped at max_ctx_tokens (the runs use 32768, the paper's largest context): appends
+    are shortened, trailing compose segments dropped;
+  * a transfer operation is, with equal probability, a state arriving from elsewhere (import of a
+    fresh segment) or a round trip of a live agent (materialize, then import of that buffer); without
+    fresh arrivals every context descends from one root and all lengths drift to the cap;
+  * compose takes 2-4 distinct live agents and releases them once their merge exists (the merged
+    branches are done), so that merging does not only ever grow the population's lengths;
+  * fork fan-out k in {1, 2, 4, 8}; new contexts go to the lowest empty slot, else they replace the
+    least recently used slot the operator does not use; an operation on an empty system is an import.
 """
 from __future__ import annotations
 
