@@ -291,6 +291,53 @@ def extra_report(args):
             out["copy_all" if copy_all else "share"] = rep
             del be
             torch.cuda.empty_cache()
+    elif args.workload == "meta":
+        # metadata-only operators: rate of back-to-back calls (host launch + device execution), against the
+        # rate of back-to-back launches of a trivial kernel on the same stream (the launch floor)
+        g = configs.Geometry(32, 8, 128, 16, 2, 4096, 64, 2048)
+        seed = configs.SEED_BASE + 2
+        be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False)
+        T = 8192
+        st, root = be.imp(be.payload(seed, 1, T), T)
+        assert st == 0
+        K = 200 * max(args.steps, 1)
+
+        def rate(fn, calls_per_iter):
+            for _ in range(20):
+                fn()
+            be.o.sync_status()
+            t0 = time.perf_counter()
+            for _ in range(K):
+                fn()
+            be.o.sync_status()  # synchronises both of the library's streams
+            dt = time.perf_counter() - t0
+            return {"calls_per_s": calls_per_iter * K / dt, "us_per_call": 1e6 * dt / (calls_per_iter * K)}
+
+        def fork_evict():
+            st, kids = be.fork(root, 16)
+            assert st == 0
+            assert be.evict(kids)[0] == 0
+
+        def fork1_evict():
+            st, kids = be.fork(root, 1)
+            assert st == 0
+            assert be.evict(kids)[0] == 0
+
+        def compose_evict():  # block-aligned segments: the merge only builds a table (1024 shared entries)
+            st, z = be.compose([root, root], 0)
+            assert st == 0
+            assert be.evict([z])[0] == 0
+
+        one = torch.zeros(1, device=dev)
+
+        def floor():
+            one.add_(1.0)
+
+        out.update({"context_blocks": T // 16,
+                    "fork16_then_evict16 (8192 + 8192 entries)": rate(fork_evict, 2),
+                    "fork1_then_evict1 (512 + 512 entries)": rate(fork1_evict, 2),
+                    "table_only_compose_then_evict (1024 entries)": rate(compose_evict, 2),
+                    "launch_floor_trivial_torch_kernel": rate(floor, 1)})
     elif args.workload == "transfer":
         # pack / unpack against host memory: one shot versus chunked with per-chunk completion flags
         g, seed, T = configs.LLAMA8B, configs.SEED_BASE + 2, 8187
@@ -400,13 +447,13 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer", "meta"])
     ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST per CTA, 2 cp.async.bulk, 3 vector LD/ST per warp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    if args.workload in ("cow", "compose", "churn", "transfer"):
+    if args.workload in ("cow", "compose", "churn", "transfer", "meta"):
         return extra_report(args)
     w = workload(args.workload)
     if args.impl == "reference":
