@@ -212,14 +212,18 @@ def extra_report(args):
         os.path.join(ROOT, "MEASURED_PEAKS.json")) else 6650.0
     out = {"workload": args.workload, "engine": args.engine, "peak_GBps": peak}
 
-    def timed(pool, fn):
-        """runs fn with kernel timing on; returns (wall ms on the stream, per-class kernel ms, bytes one way)"""
+    def timed(pool, fn, meta=False):
+        """runs fn with kernel timing on; returns (ms on the stream, per-class kernel ms, bytes one way).
+        meta=True: fn is a metadata-only operator, which runs on the library's own stream; the host then waits
+        for both of the library's streams before the closing event, so ms is the call's wall time."""
         s0 = pool.stats()
         pool.set_timing(True)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
         fn()
+        if meta:
+            pool.sync_status()
         e1.record()
         torch.cuda.synchronize()
         pool.set_timing(False)
@@ -240,11 +244,11 @@ def extra_report(args):
         for it in range(args.warmup + args.steps):
             st, root = be.imp(root_buf, T)
             res = {}
-            ms_f, _, _ = timed(be.o, lambda: res.update(r=be.fork(root, kids_n)))
+            ms_f, _, _ = timed(be.o, lambda: res.update(r=be.fork(root, kids_n)), meta=True)
             kids = res["r"][1]
             ms_a, dms, b = timed(be.o, lambda: res.update(a=be.append(kids, [1] * kids_n, one)[0]))
             assert res["a"] == 0
-            ms_e, _, _ = timed(be.o, lambda: res.update(e=(be.evict(kids)[0], be.evict([root])[0])))
+            ms_e, _, _ = timed(be.o, lambda: res.update(e=(be.evict(kids)[0], be.evict([root])[0])), meta=True)
             assert res["r"][0] == 0 and res["e"] == (0, 0), res
             if it >= args.warmup:
                 acc["append_ms"] += dms["append"]; acc["append_bytes"] += b
