@@ -52,6 +52,10 @@ def workload(name: str):
         g = configs.LLAMA8B
         return dict(name="llama3-8b-shaped KV, 8187-token context, 16 agents x 512 tokens, unaligned (COW)", g=g,
                     seed=configs.SEED_BASE + 2, T=8187, agents=16, n_new=512)
+    if name == "8b-aligned":  # the literal block-aligned variant: no copy-on-write, the compose is table-only
+        g = configs.LLAMA8B
+        return dict(name="llama3-8b-shaped KV, 8192-token context, 16 agents x 512 tokens, block-aligned", g=g,
+                    seed=configs.SEED_BASE + 2, T=8192, agents=16, n_new=512)
     if name == "70b":
         g = configs.LLAMA70B
         return dict(name="llama3-70b-shaped KV, 32763-token context, 8 agents x 1024 tokens, unaligned (COW)", g=g,
@@ -451,7 +455,7 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="8b", choices=["8b", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer", "meta"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "8b-aligned", "70b", "8b-small", "tiny", "cow", "compose", "churn", "transfer", "meta"])
     ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST per CTA, 2 cp.async.bulk, 3 vector LD/ST per warp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
