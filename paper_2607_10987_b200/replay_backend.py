@@ -36,7 +36,9 @@ class GpuBackend:
         self.o = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, g.n_blocks, g.max_ctx,
                         g.max_blocks_per_ctx, free_order=free_order, max_batch=max_batch)
         self.o.set_copy_engine(engine)
-        if init_fill:
+        if init_fill == "zero":  # all-zero pool image (matches a freshly created oracle pool)
+            self.o.pool.zero_()
+        elif init_fill:
             fill.fill_torch(seed, 0, 0, g.pool_bytes // 2, self.o.device, out=self.o.pool.view(torch.int16))
         self.staging = (torch.empty(staging_tokens * g.bpt, dtype=torch.uint8, device=self.o.device)
                         if staging_tokens else None)

@@ -24,7 +24,7 @@ class OracleBackend:
         self.layers = list(range(g.n_layers)) if layers is None else list(layers)
         self.o = paged.PagedOracle(len(self.layers), g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes,
                                    g.n_blocks, g.max_ctx, g.max_blocks_per_ctx, free_order)
-        if init_fill:
+        if init_fill and init_fill != "zero":  # "zero": keep the all-zero image the oracle starts with
             pv = self.o.pool_view()
             per_layer = g.layer_stride // 2  # elements
             step = 1 << 24  # elements per chunk: keeps the generator's temporaries small

@@ -28,7 +28,9 @@ def test_config2_llama8b_full_pool(unaligned):
     g, seed, ops = configs.config2(unaligned)
     if not _fits(g, 12):
         pytest.skip("not enough free device memory for the 64 GiB pool")
-    gpu, cpu = lockstep(g, seed, ops, layers=[0, g.n_layers - 1])
+    # unaligned variant: seeded pool image, two layers compared; literal variant: zero image, one layer
+    gpu, cpu = (lockstep(g, seed, ops, layers=[0, g.n_layers - 1]) if unaligned else
+                lockstep(g, seed, ops, layers=[g.n_layers // 2], init_fill="zero"))
     st = gpu.o.stats()
     assert st["cow_count"] == (16 if unaligned else 0)
     assert st["live_blocks"] == (512 + 512 + 16 * 32 + (16 if unaligned else 0))
@@ -52,7 +54,7 @@ def test_config3_compose_levels_8b(copy_all):
     g, seed, ops, lens = configs.config3(configs.LLAMA8B, copy_all=copy_all)
     if not _fits(g, 16):
         pytest.skip("not enough free device memory for the 64 GiB pool")
-    gpu, cpu = lockstep(g, seed, ops, layers=[3, 30])
+    gpu, cpu = lockstep(g, seed, ops, layers=[30] if copy_all else [3], init_fill="zero")
     assert gpu.o.ctx_len(gpu.o.live_ctxs()[-1]) == sum(lens)
 
 

@@ -27,12 +27,12 @@ def same_catalog_export(gpu, cpu):
         assert got[k].dtype == want[k].dtype and np.array_equal(got[k], want[k]), k
 
 
-def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None):
+def lockstep(g, seed, ops, layers=None, engine=0, max_batch=0, order=None, init_fill=True):
     """Replays ops on the GPU library and on the oracle side by side and compares after every op."""
     layers = list(range(g.n_layers)) if layers is None else list(layers)
     order = configs.free_order(seed, g.n_blocks) if order is None else order
-    gpu = GpuBackend(g, seed, free_order=order, engine=engine, max_batch=max_batch)
-    cpu = OracleBackend(g, seed, layers=layers, free_order=order)
+    gpu = GpuBackend(g, seed, free_order=order, engine=engine, max_batch=max_batch, init_fill=init_fill)
+    cpu = OracleBackend(g, seed, layers=layers, free_order=order, init_fill=init_fill)
     for (i, op, st_g, res_g, _), (_, _, st_c, res_c, _) in zip(replay(ops, gpu, seed), replay(ops, cpu, seed)):
         assert st_g == st_c, (i, op, st_g, st_c)
         assert gpu.snapshot() == cpu.snapshot(), (i, op)
