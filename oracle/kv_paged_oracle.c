@@ -58,6 +58,11 @@ typedef struct kvo_pool {
     int64_t *reuse;       /* [max_ctx] times the state was read by fork / materialize / compose   */
     int64_t *last_access; /* [max_ctx] logical clock of the last operator that used the state     */
     int64_t clock;        /* logical clock: number of successful state-touching operators so far  */
+    /* lineage Lambda (Sec. 3.2: how a state was produced; App. A.2 catalog field "lineage") */
+    int32_t *origin;      /* [max_ctx] 1 = registered from a buffer (prefill / transfer), 2 = fork, 3 = merge */
+    int32_t *parent;      /* [max_ctx] handle the state descends from (fork parent, first merged segment), -1 = none */
+    int64_t *born;        /* [max_ctx] clock of the operator that created the state               */
+    int64_t *parent_born; /* [max_ctx] creation clock of that parent: (handle, born) names a state for good */
     int64_t peak_live;    /* max over time of NB - free (Mem_KV in blocks, Sec. 6.2) */
     int64_t cow_count;    /* copy-on-write events so far              */
     int64_t rows_copied;  /* rows moved by memcpy so far              */
@@ -132,7 +137,14 @@ static int has_duplicates(const int32_t *v, int32_t n) {
 /* Catalog bookkeeping (metadata catalog of App. A.2: "last_access: timestamp or logical clock for
  * eviction"; the reuse term of the eviction score).  The logical clock counts successful
  * state-touching operators; an operator stamps every state it reads, writes or creates. */
-static void born(kvo_pool *p, int32_t c) { p->reuse[c] = 0; p->last_access[c] = p->clock; }
+static void born(kvo_pool *p, int32_t c, int32_t origin, int32_t parent) {
+    p->reuse[c] = 0;
+    p->last_access[c] = p->clock;
+    p->born[c] = p->clock;
+    p->origin[c] = origin;
+    p->parent[c] = parent;
+    p->parent_born[c] = parent >= 0 ? p->born[parent] : -1;
+}
 static void read_by_other(kvo_pool *p, int32_t c) { p->reuse[c] += 1; p->last_access[c] = p->clock; }
 
 /* ---------------------------------------------------------------- create / destroy */
@@ -155,7 +167,13 @@ kvo_pool *kvo_create(int32_t L, int32_t H, int32_t D, int32_t BS, int32_t E, int
     p->len = (int64_t *)malloc((size_t)max_ctx * sizeof(int64_t));
     p->reuse = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
     p->last_access = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
-    if (!p->pool || !p->refcount || !p->ring || !p->table || !p->len || !p->reuse || !p->last_access) return NULL;
+    p->origin = (int32_t *)calloc((size_t)max_ctx, sizeof(int32_t));
+    p->parent = (int32_t *)calloc((size_t)max_ctx, sizeof(int32_t));
+    p->born = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
+    p->parent_born = (int64_t *)calloc((size_t)max_ctx, sizeof(int64_t));
+    if (!p->pool || !p->refcount || !p->ring || !p->table || !p->len || !p->reuse || !p->last_access || !p->origin ||
+        !p->parent || !p->born || !p->parent_born)
+        return NULL;
     for (int32_t i = 0; i < NB; ++i) p->ring[i] = free_order ? free_order[i] : i;
     for (int32_t c = 0; c < max_ctx; ++c) p->len[c] = -1;
     p->head = 0;
@@ -166,7 +184,7 @@ kvo_pool *kvo_create(int32_t L, int32_t H, int32_t D, int32_t BS, int32_t E, int
 void kvo_destroy(kvo_pool *p) {
     if (!p) return;
     free(p->pool); free(p->refcount); free(p->ring); free(p->table); free(p->len);
-    free(p->reuse); free(p->last_access);
+    free(p->reuse); free(p->last_access); free(p->origin); free(p->parent); free(p->born); free(p->parent_born);
     free(p);
 }
 
@@ -181,6 +199,10 @@ kvo_pool *kvo_clone(const kvo_pool *s) {
     memcpy(p->len, s->len, (size_t)s->max_ctx * sizeof(int64_t));
     memcpy(p->reuse, s->reuse, (size_t)s->max_ctx * sizeof(int64_t));
     memcpy(p->last_access, s->last_access, (size_t)s->max_ctx * sizeof(int64_t));
+    memcpy(p->origin, s->origin, (size_t)s->max_ctx * sizeof(int32_t));
+    memcpy(p->parent, s->parent, (size_t)s->max_ctx * sizeof(int32_t));
+    memcpy(p->born, s->born, (size_t)s->max_ctx * sizeof(int64_t));
+    memcpy(p->parent_born, s->parent_born, (size_t)s->max_ctx * sizeof(int64_t));
     p->clock = s->clock;
     p->head = s->head; p->tail = s->tail;
     p->peak_live = s->peak_live; p->cow_count = s->cow_count; p->rows_copied = s->rows_copied;
@@ -208,7 +230,7 @@ int kvo_import(kvo_pool *p, const void *buf, int64_t n, int32_t *out_ctx) {
     for (int64_t tok = 0; tok < n; ++tok) store_token(p, t, tok, buf, n, tok);
     p->len[c] = n;
     p->clock += 1;
-    born(p, c);
+    born(p, c, 1, -1);
     *out_ctx = c;
     return KVO_OK;
 }
@@ -260,7 +282,7 @@ int kvo_fork(kvo_pool *p, int32_t parent, int32_t k, int32_t *out_children) {
             p->refcount[tbl(p, parent)[q]] += 1;
         }
         p->len[c] = p->len[parent];
-        born(p, c);
+        born(p, c, 2, parent);
         out_children[j] = c;
     }
     return KVO_OK;
@@ -382,7 +404,7 @@ int kvo_compose(kvo_pool *p, int32_t m, const int32_t *segs, uint32_t flags, int
         off += T;
     }
     p->len[c] = off;
-    born(p, c);
+    born(p, c, 3, segs[0]);
     *out_ctx = c;
     return KVO_OK;
 }
@@ -446,12 +468,13 @@ int kvo_evict_to_budget(kvo_pool *p, double alpha, double beta, double gamma, in
 
 /* Columnar export of the metadata catalog (App. A.2, table of catalog fields; Sec. 5.3: metadata in a
  * columnar, zero-copy encoding).  State rows: one per live state in ascending handle order
- * (state_id, n_tokens, reuse, last_access) plus list offsets into the block rows (offsets[i] =
+ * (state_id, n_tokens, reuse, last_access, lineage: origin, parent, born, parent_born) plus list offsets into the block rows (offsets[i] =
  * number of block rows of the states before i, offsets[n_states] = total); block rows: one per
  * block-table entry (block_id, position range [pos_begin, pos_end) within the state, refcount of the
  * block, byte address of the block's layer-0 K run relative to the pool base).  Returns the counts. */
 int kvo_export_catalog(const kvo_pool *p, int32_t *state_id, int64_t *n_tokens, int64_t *reuse,
-                       int64_t *last_access, int32_t *block_offsets, int32_t *block_id, int64_t *pos_begin,
+                       int64_t *last_access, int32_t *origin, int32_t *parent, int64_t *born_at,
+                       int64_t *parent_born, int32_t *block_offsets, int32_t *block_id, int64_t *pos_begin,
                        int64_t *pos_end, int32_t *refcount, int64_t *address, int32_t *n_states,
                        int32_t *n_block_rows) {
     int32_t ns = 0, nr = 0;
@@ -461,6 +484,10 @@ int kvo_export_catalog(const kvo_pool *p, int32_t *state_id, int64_t *n_tokens, 
         n_tokens[ns] = p->len[c];
         reuse[ns] = p->reuse[c];
         last_access[ns] = p->last_access[c];
+        origin[ns] = p->origin[c];
+        parent[ns] = p->parent[c];
+        born_at[ns] = p->born[c];
+        parent_born[ns] = p->parent_born[c];
         block_offsets[ns] = nr;
         for (int64_t j = 0; j < nblk(p, p->len[c]); ++j) {
             int32_t b = tbl(p, c)[j];

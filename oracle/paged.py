@@ -18,6 +18,7 @@ _LIB = os.path.join(_HERE, "libkvoracle.so")
 
 OK, INVALID_ARG, BAD_CTX, OOM_BLOCKS, OOM_CTX, TOO_LONG, DST_TOO_SMALL = 0, -1, -2, -3, -4, -5, -7
 COMPOSE_COPY_ALL = 1
+STATE_COLUMNS = ("state_id", "n_tokens", "reuse", "last_access", "origin", "parent", "born", "parent_born")
 
 _lib = None
 
@@ -60,7 +61,7 @@ def lib():
         L.kvo_stats.argtypes = [vp, p64]
         L.kvo_evict_to_budget.argtypes = [vp, C.c_double, C.c_double, C.c_double, i64, p32, i32, p32]
         L.kvo_get_catalog.argtypes = [vp, p64, p64, p64]
-        L.kvo_export_catalog.argtypes = [vp, p32, p64, p64, p64, p32, p32, p64, p64, p32, p64, p32, p32]
+        L.kvo_export_catalog.argtypes = [vp, p32, p64, p64, p64, p32, p32, p64, p64, p32, p32, p64, p64, p32, p64, p32, p32]
         _lib = L
     return _lib
 
@@ -174,19 +175,20 @@ class PagedOracle:
         i32 = lambda n: np.zeros(n, dtype=np.int32)
         i64 = lambda n: np.zeros(n, dtype=np.int64)
         cols = {"state_id": i32(self.max_ctx), "n_tokens": i64(self.max_ctx), "reuse": i64(self.max_ctx),
-                "last_access": i64(self.max_ctx), "block_offsets": i32(self.max_ctx + 1), "block_id": i32(cap_rows),
+                "last_access": i64(self.max_ctx), "origin": i32(self.max_ctx), "parent": i32(self.max_ctx),
+                "born": i64(self.max_ctx), "parent_born": i64(self.max_ctx),
+                "block_offsets": i32(self.max_ctx + 1), "block_id": i32(cap_rows),
                 "pos_begin": i64(cap_rows), "pos_end": i64(cap_rows), "refcount": i32(cap_rows),
                 "address": i64(cap_rows)}
         ns, nr = C.c_int32(0), C.c_int32(0)
         P32, P64 = C.POINTER(C.c_int32), C.POINTER(C.c_int64)
         ptr = lambda k: cols[k].ctypes.data_as(P32 if cols[k].dtype == np.int32 else P64)
         lib().kvo_export_catalog(self.h, ptr("state_id"), ptr("n_tokens"), ptr("reuse"), ptr("last_access"),
-                                 ptr("block_offsets"), ptr("block_id"), ptr("pos_begin"), ptr("pos_end"),
+                                 ptr("origin"), ptr("parent"), ptr("born"), ptr("parent_born"), ptr("block_offsets"), ptr("block_id"), ptr("pos_begin"), ptr("pos_end"),
                                  ptr("refcount"), ptr("address"), C.byref(ns), C.byref(nr))
         out = {}
         for k, v in cols.items():
-            n = ns.value + 1 if k == "block_offsets" else (ns.value if k in ("state_id", "n_tokens", "reuse",
-                                                                             "last_access") else nr.value)
+            n = ns.value + 1 if k == "block_offsets" else (ns.value if k in STATE_COLUMNS else nr.value)
             out[k] = v[:n].copy()
         return out
 

@@ -632,3 +632,21 @@ def test_catalog_export_of_an_empty_pool():
     o = small_pool()
     cols = o.export_catalog()
     assert cols["state_id"].size == 0 and cols["block_offsets"].tolist() == [0] and cols["block_id"].size == 0
+
+
+def test_catalog_lineage_columns():
+    """Lineage (how a state was produced, from which state): hand-derived for the sequence of _busy_pool:
+    import a (clock 1), import b (2), fork a -> 2,3,4 (3), ..., compose [kid1, b] -> 5 (7)."""
+    o, rng = _busy_pool()
+    cols = o.export_catalog()
+    assert cols["origin"].tolist() == [1, 1, 2, 2, 2, 3]          # 1 registered buffer, 2 fork, 3 merge
+    assert cols["parent"].tolist() == [-1, -1, 0, 0, 0, 3]        # fork parent / first merged segment
+    assert cols["born"].tolist() == [1, 2, 3, 3, 3, 7]
+    assert cols["parent_born"].tolist() == [-1, -1, 1, 1, 1, 3]
+    # a handle is reused after eviction; (handle, born) still tells the two states apart
+    o.evict([0])                                                  # clock 10
+    c = o.imp(rand_buf(rng, o, 3), 3)[1]                          # clock 11, takes handle 0 again
+    assert c == 0
+    cols = o.export_catalog()
+    assert cols["born"].tolist()[0] == 11 and cols["origin"].tolist()[0] == 1
+    assert cols["parent"].tolist()[2:5] == [0, 0, 0] and cols["parent_born"].tolist()[2:5] == [1, 1, 1]
