@@ -257,17 +257,25 @@ int aaf_kv_get_free_list(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entrie
  * can wrap them without conversion.
  *   state rows, one per live context in ascending handle order (capacity max_ctx):
  *     state_id int32, n_tokens int64, reuse int64, last_access int64,
+ *     lineage (Lambda of Sec. 3.2): origin int32 (AAF_ORIGIN_*), parent int32 (the fork parent or the
+ *     first merged segment, -1 for none), born int64 (clock of the creating call), parent_born int64
+ *     (creation clock of that parent: handles are reused, (handle, born) names a state for good),
  *     block_offsets int32[n_states + 1]: list offsets into the block rows (exclusive prefix sum of
  *     the block-table lengths; capacity max_ctx + 1)
  *   block rows, one per block-table entry (capacity = n_block_rows of aaf_kv_catalog_rows):
  *     block_id int32, pos_begin / pos_end int64 (token range within the context), refcount int32,
  *     address int64 (byte offset of the block's layer-0 K run from pool_base; layer l and V follow
  *     by + l * layer_stride_bytes and + run).
- * model_id / config_hash (M, Theta) are pool-wide and live in the pool descriptor; lineage, device
- * and owner are the caller's tags.  aaf_kv_catalog_rows answers from the host mirror (no sync). */
+ * model_id / config_hash (M, Theta) are pool-wide and live in the pool descriptor; device and owner
+ * are the caller's tags.  aaf_kv_catalog_rows answers from the host mirror (no sync). */
+#define AAF_ORIGIN_BUFFER 1 /* registered from a transfer buffer: prefill output or received state */
+#define AAF_ORIGIN_FORK 2
+#define AAF_ORIGIN_MERGE 3
 typedef struct aaf_kv_catalog_cols {
     int32_t *state_id;
     int64_t *n_tokens, *reuse, *last_access;
+    int32_t *origin, *parent;
+    int64_t *born, *parent_born;
     int32_t *block_offsets;
     int32_t *block_id;
     int64_t *pos_begin, *pos_end;

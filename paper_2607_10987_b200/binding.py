@@ -58,6 +58,7 @@ class aaf_kv_stats(C.Structure):
 
 class aaf_kv_catalog_cols(C.Structure):
     _fields_ = [("state_id", C.c_void_p), ("n_tokens", C.c_void_p), ("reuse", C.c_void_p), ("last_access", C.c_void_p),
+                ("origin", C.c_void_p), ("parent", C.c_void_p), ("born", C.c_void_p), ("parent_born", C.c_void_p),
                 ("block_offsets", C.c_void_p), ("block_id", C.c_void_p), ("pos_begin", C.c_void_p),
                 ("pos_end", C.c_void_p), ("refcount", C.c_void_p), ("address", C.c_void_p)]
 
@@ -322,6 +323,7 @@ class KVPool:
         i32 = lambda n: torch.empty(max(n, 1), dtype=torch.int32, device=self.device)
         i64 = lambda n: torch.empty(max(n, 1), dtype=torch.int64, device=self.device)
         t = {"state_id": i32(ns.value), "n_tokens": i64(ns.value), "reuse": i64(ns.value), "last_access": i64(ns.value),
+             "origin": i32(ns.value), "parent": i32(ns.value), "born": i64(ns.value), "parent_born": i64(ns.value),
              "block_offsets": i32(ns.value + 1), "block_id": i32(nr.value), "pos_begin": i64(nr.value),
              "pos_end": i64(nr.value), "refcount": i32(nr.value), "address": i64(nr.value)}
         cols = aaf_kv_catalog_cols(**{k: v.data_ptr() for k, v in t.items()})
@@ -329,7 +331,8 @@ class KVPool:
         if st != AAF_OK:
             raise RuntimeError(aaf_kv_strerror(st))
         n_of = lambda k: ns.value + 1 if k == "block_offsets" else (
-            ns.value if k in ("state_id", "n_tokens", "reuse", "last_access") else nr.value)
+            ns.value if k in ("state_id", "n_tokens", "reuse", "last_access", "origin", "parent", "born",
+                              "parent_born") else nr.value)
         return {k: v[: n_of(k)] for k, v in t.items()}
 
     def materialize_host_chunked(self, ctx, t0, t1, dst_host, staging, chunk_tokens, flags=None):

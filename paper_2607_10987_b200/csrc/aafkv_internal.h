@@ -57,6 +57,11 @@ struct DevState {
     unsigned long long *cat_reuse;
     long long *cat_last;
     double *cat_score;  // scratch of the scored eviction
+    // lineage per handle: how the state was produced (1 buffer, 2 fork, 3 merge), from which handle, when
+    int *cat_origin;
+    int *cat_parent;
+    long long *cat_born;
+    long long *cat_parent_born;
 };
 
 // ---- per-call argument records (written by the host into pinned memory, read by planners)

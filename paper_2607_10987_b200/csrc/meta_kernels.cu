@@ -59,6 +59,19 @@ __device__ __forceinline__ void add_payload(DevCtl *ctl, unsigned long long byte
     if ((threadIdx.x & 31) == 0 && bytes) atomicAdd(&ctl->payload_bytes, bytes);
 }
 
+// Catalog entry of a state that has just been created (lineage: origin 1 = registered from a buffer,
+// 2 = fork, 3 = merge; parent = handle it descends from or -1).
+__device__ __forceinline__ void catalog_born(const DevState &s, int c, long long len, long long clock, int origin,
+                                             int parent) {
+    s.cat_len[c] = len;
+    s.cat_reuse[c] = 0;
+    s.cat_last[c] = clock;
+    s.cat_origin[c] = origin;
+    s.cat_parent[c] = parent;
+    s.cat_born[c] = clock;
+    s.cat_parent_born[c] = parent >= 0 ? s.cat_born[parent] : -1;
+}
+
 // Argument records arrive in pinned host memory that the kernel reads over PCIe; every such read costs
 // a bus round trip and is not cached, so a kernel that searches its records stages them first: one
 // coalesced pass into shared memory (when they fit), then all further reads are on-chip.
@@ -156,11 +169,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevSt
             s.ctl->head = head0 + nblk;
             note_alloc(s.ctl, g, head0 + nblk, tail);
             s.ctl->payload_bytes += (unsigned long long)(n * 2 * g.L * g.row);
-            if (s.cat_len) {
-                s.cat_len[ctx] = n;
-                s.cat_reuse[ctx] = 0;
-                s.cat_last[ctx] = clock;
-            }
+            if (s.cat_len) catalog_born(s, ctx, n, clock, 1, -1);
         }
     }
 }
@@ -181,9 +190,7 @@ __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int paren
         s.tables[(long long)children[q] * g.max_blk + j] = b;
         if (q == 0) atomicAdd(&s.refcount[b], k);
         if (j == 0 && s.cat_len) {  // catalog: the child is born, the parent was read
-            s.cat_len[children[q]] = T;
-            s.cat_reuse[children[q]] = 0;
-            s.cat_last[children[q]] = clock;
+            catalog_born(s, children[q], T, clock, 2, parent);
             if (q == 0) {
                 s.cat_reuse[parent] += 1;
                 s.cat_last[parent] = clock;
@@ -409,11 +416,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
         } else {
             s.ctl->head = head0 + total_fresh;
             note_alloc(s.ctl, g, head0 + total_fresh, tail);
-            if (s.cat_len) {
-                s.cat_len[out_ctx] = segs[m - 1].off + segs[m - 1].T;
-                s.cat_reuse[out_ctx] = 0;
-                s.cat_last[out_ctx] = clock;
-            }
+            if (s.cat_len) catalog_born(s, out_ctx, segs[m - 1].off + segs[m - 1].T, clock, 3, segs[0].ctx);
         }
     }
 }
@@ -650,6 +653,10 @@ __global__ void __launch_bounds__(PLAN_THREADS) export_states_kernel(Geom g, Dev
             cols.n_tokens[row] = len;
             cols.reuse[row] = (long long)s.cat_reuse[c];
             cols.last_access[row] = s.cat_last[c];
+            cols.origin[row] = s.cat_origin[c];
+            cols.parent[row] = s.cat_parent[c];
+            cols.born[row] = s.cat_born[c];
+            cols.parent_born[row] = s.cat_parent_born[c];
             cols.block_offsets[row] = off;
         }
         row_carry += live_tot;

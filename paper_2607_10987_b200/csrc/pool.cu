@@ -27,7 +27,7 @@ namespace {
 constexpr int ARG_SLOTS = 16;
 
 struct Layout {
-    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, total;
+    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, cat_origin, cat_parent, cat_born, cat_parent_born, total;
     int max_pieces, max_batch;
 };
 
@@ -60,6 +60,10 @@ Layout make_layout(const aaf_kv_pool_desc *d) {
     L.cat_reuse = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
     L.cat_last = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
     L.cat_score = off; off = align_up(off + sizeof(double) * (size_t)d->max_ctx, 256);
+    L.cat_origin = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx, 256);
+    L.cat_parent = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx, 256);
+    L.cat_born = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
+    L.cat_parent_born = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
     L.total = off;
     return L;
 }
@@ -400,6 +404,10 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     p->s.cat_reuse = reinterpret_cast<unsigned long long *>(ws + lay.cat_reuse);
     p->s.cat_last = reinterpret_cast<long long *>(ws + lay.cat_last);
     p->s.cat_score = reinterpret_cast<double *>(ws + lay.cat_score);
+    p->s.cat_origin = reinterpret_cast<int *>(ws + lay.cat_origin);
+    p->s.cat_parent = reinterpret_cast<int *>(ws + lay.cat_parent);
+    p->s.cat_born = reinterpret_cast<long long *>(ws + lay.cat_born);
+    p->s.cat_parent_born = reinterpret_cast<long long *>(ws + lay.cat_parent_born);
     p->len.assign((size_t)desc->max_ctx, -1);
     p->free_lb = desc->n_blocks;
 
@@ -854,7 +862,8 @@ int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void 
     int32_t ns = 0;
     int64_t rows = 0;
     aaf_kv_catalog_rows(p, &ns, &rows);
-    if (!cols->state_id || !cols->n_tokens || !cols->reuse || !cols->last_access || !cols->block_offsets)
+    if (!cols->state_id || !cols->n_tokens || !cols->reuse || !cols->last_access || !cols->block_offsets ||
+        !cols->origin || !cols->parent || !cols->born || !cols->parent_born)
         return AAF_ERR_INVALID_ARG;
     if (rows > 0 && (!cols->block_id || !cols->pos_begin || !cols->pos_end || !cols->refcount || !cols->address))
         return AAF_ERR_INVALID_ARG;
