@@ -42,9 +42,10 @@ from workloads import configs, fill  # noqa: E402
 METRIC = "kv_bytes_moved_GBps"
 UNIT = "GB/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per algorithmic byte for the copy kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists)
-TRAFFIC_PER_ALGORITHMIC_BYTE = 0.90  # profiles/copy_bulk_kernel_8b-small_ncu_full.md: (267.9 + 216.4) / (2 x 267.8) MB
+# dram__bytes_read.sum + dram__bytes_write.sum per algorithmic byte for the copy kernel, from the one-pass ncu
+# capture of the full-size launches summarised in profiles/copy_bulk_kernel_8b_dram_bytes.md:
+# (5.440 + 5.219) GB of DRAM traffic for 10.915 GB algorithmic (read + written) over the five launches of a step
+TRAFFIC_PER_ALGORITHMIC_BYTE = 0.977
 
 
 def workload(name: str):
