@@ -206,8 +206,8 @@ int aaf_kv_evict(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, void *stre
  * operation.  While the live blocks (n_blocks - free) exceed budget_blocks, the context with the
  * lowest score (ties: smallest handle) is evicted by the release rule of aaf_kv_evict.  Shared
  * blocks survive while another context references them.  out_victims (host, cap >= number of live
- * contexts) receives the evicted handles in order, *n_victims their count.  The call synchronises
- * `stream` (the host needs the victims).  alpha = beta = 0, gamma > 0 is LRU.
+ * contexts) receives the evicted handles in order, *n_victims their count.  The call waits for the
+ * metadata kernels issued so far, not for copies still running on `stream` (the host needs the victims).  alpha = beta = 0, gamma > 0 is LRU.
  * Errors: INVALID_ARG (negative budget, non-finite weight, cap too small), CUDA. */
 int aaf_kv_evict_to_budget(aaf_kv_pool *pool, double alpha, double beta, double gamma, int64_t budget_blocks,
                            aaf_ctx_t *out_victims, int32_t cap, int32_t *n_victims, void *stream);
@@ -246,15 +246,16 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *pool, const void *src_host, const aa
                                void *staging_dev, size_t staging_bytes, int32_t chunk_tokens, aaf_ctx_t *out_ctx,
                                void *stream);
 
-/* Introspection (metadata catalog of App. A.2).  These synchronise the pool's stream. */
+/* Introspection (metadata catalog of App. A.2).  These synchronise the library's metadata stream and
+ * the stream of the most recent call. */
 int aaf_kv_ctx_len(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t *n_tokens);
 int aaf_kv_get_table(aaf_kv_pool *pool, aaf_ctx_t ctx, int32_t *host_out, int32_t cap, int32_t *n_blocks);
 int aaf_kv_get_refcounts(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */);
 int aaf_kv_get_free_list(aaf_kv_pool *pool, int32_t *host_out /* n_blocks entries */, int32_t *n_free);
 /* Columnar export of the metadata catalog (App. A.2, catalog fields; Sec. 5.3: metadata kept in a
  * columnar, zero-copy encoding).  All columns are DEVICE buffers the caller owns; they are written
- * by kernels on `stream` and are laid out like Arrow primitive arrays and list offsets, so a consumer
- * can wrap them without conversion.
+ * by metadata kernels that `stream` is made to wait for, and are laid out like Arrow primitive arrays
+ * and list offsets, so a consumer on `stream` can wrap them without conversion.
  *   state rows, one per live context in ascending handle order (capacity max_ctx):
  *     state_id int32, n_tokens int64, reuse int64, last_access int64,
  *     lineage (Lambda of Sec. 3.2): origin int32 (AAF_ORIGIN_*), parent int32 (the fork parent or the
