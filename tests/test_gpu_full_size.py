@@ -78,3 +78,13 @@ def test_cow_stress_1024_children_8b_rows():
     st = gpu.o.stats()
     assert st["cow_count"] == 1024
     assert st["live_blocks"] == 512 + 1024
+    # one batched evict of all 1024 children (525 K table entries on 1.5 K blocks): the large-batch path
+    # (release over a grid, compaction afterwards) must free the same blocks in the same order
+    kids = [c for c in cpu.o.live_ctxs() if c != 0]
+    assert len(kids) == 1024
+    assert gpu.evict(kids)[0] == 0 and cpu.evict(kids)[0] == 0
+    assert gpu.snapshot() == cpu.snapshot()
+    assert gpu.o.stats()["live_blocks"] == 512
+    assert gpu.evict([0])[0] == 0 and cpu.evict([0])[0] == 0
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+    assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
