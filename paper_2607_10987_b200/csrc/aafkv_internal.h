@@ -33,7 +33,8 @@ struct DevCtl {
     unsigned long long probe_need;     // dry-run result of the append planner
     unsigned int one;                  // constant 1: source of the host-visible chunk completion flags
     unsigned int pad32;
-    unsigned long long pad[8];
+    unsigned long long evict_tail0;    // ring tail before the current large evict (read by its scatter kernel)
+    unsigned long long pad[7];
 };
 static_assert(sizeof(DevCtl) == 128, "DevCtl layout");
 
@@ -52,6 +53,7 @@ struct DevState {
     int *tables;     // [max_ctx][max_blk]
     Piece *pieces;   // [max_pieces]
     int *scratch;    // [3 * max_batch] per-batch scratch of the append planner
+    int *tile_count; // [max_ctx * max_blk / 8192 + 2] per-tile counts / offsets of a large evict
     // metadata catalog per handle (App. A.2): tokens (-1 = free handle), reads by other states, last access
     long long *cat_len;
     unsigned long long *cat_reuse;

@@ -431,10 +431,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
 //   The mark's high 32 bits are the call's logical clock, so marks of earlier calls are always
 //   smaller and the mark array never needs clearing.
 //   Small batches (<= EVICT_FUSED_MAX entries) run both phases in one CTA; larger ones run the release
-//   over a grid and the compaction in one CTA.
-constexpr int EVICT_STAGE = 2048;        // ints staged in shared memory: ctx[n] followed by ent_off[n + 1]
+//   over a grid and the compaction as count / scan / scatter over tiles.
+constexpr int EVICT_STAGE = 2064;        // ints staged in shared memory: ctx[n] followed by ent_off[n + 1] (n <= 1031)
 constexpr int EVICT_ITEMS = 8;           // consecutive flattened entries per thread and pass
 constexpr int EVICT_FUSED_MAX = 32768;
+constexpr int EVICT_TILE = 1024 * EVICT_ITEMS;  // entries per CTA and pass (PLAN_THREADS threads)
 
 __device__ __forceinline__ int find_ctx_index(const int *ent_off, int n, int e) {
     int lo = 0, hi = n - 1;  // last context whose first entry is <= e
@@ -453,56 +454,124 @@ __device__ __forceinline__ void evict_release_entry(const Geom &g, const DevStat
     atomicMax(&s.last_pos[b], stamp | (unsigned long long)(unsigned)e);
 }
 
+// One thread's share of a tile: its EVICT_ITEMS consecutive entries starting at e0.  Fills blk[] and
+// returns the bit mask of the entries that free their block (count reached 0 and this entry is the
+// block's last occurrence in the batch).  Reads only; the same call gives the same answer in every
+// kernel that runs after the release phase.
+__device__ __forceinline__ unsigned evict_thread_flags(const Geom &g, const DevState &s, const int *ctx,
+                                                       const int *ent_off, int n, int total, int e0,
+                                                       unsigned long long stamp, int (&blk)[EVICT_ITEMS]) {
+    // locate the first entry once, then walk (context, position) forward: all table reads are independent
+    int ci = e0 < total ? find_ctx_index(ent_off, n, e0) : 0;
+#pragma unroll
+    for (int k = 0; k < EVICT_ITEMS; ++k) {
+        const int e = e0 + k;
+        blk[k] = -1;
+        if (e < total) {
+            while (e >= ent_off[ci + 1]) ++ci;
+            blk[k] = s.tables[(long long)ctx[ci] * g.max_blk + (e - ent_off[ci])];
+        }
+    }
+    int rc[EVICT_ITEMS];
+    unsigned long long lp[EVICT_ITEMS];
+#pragma unroll
+    for (int k = 0; k < EVICT_ITEMS; ++k) {
+        rc[k] = blk[k] >= 0 ? s.refcount[blk[k]] : 1;
+        lp[k] = blk[k] >= 0 ? s.last_pos[blk[k]] : 0ull;
+    }
+    unsigned flags = 0;
+#pragma unroll
+    for (int k = 0; k < EVICT_ITEMS; ++k) {
+        const bool f = blk[k] >= 0 && rc[k] == 0 && lp[k] == (stamp | (unsigned long long)(unsigned)(e0 + k));
+        flags |= (f ? 1u : 0u) << k;
+    }
+    return flags;
+}
+
+__device__ __forceinline__ void evict_write_ring(const Geom &g, const DevState &s, unsigned long long tail0, int pos,
+                                                 unsigned flags, const int (&blk)[EVICT_ITEMS]) {
+#pragma unroll
+    for (int k = 0; k < EVICT_ITEMS; ++k)
+        if (flags & (1u << k)) {
+            s.ring[(tail0 + (unsigned long long)pos) % (unsigned long long)g.NB] = blk[k];
+            ++pos;
+        }
+}
+
+__device__ __forceinline__ void evict_finish(const Geom &g, const DevState &s, const int *ctx, int n,
+                                             unsigned long long tail0, int freed) {
+    if (s.cat_len)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) s.cat_len[ctx[i]] = -1;
+    if (threadIdx.x == 0) {
+        if (tail0 + freed - s.ctl->head > (unsigned long long)g.NB) set_status(s.ctl, AAF_ERR_CORRUPT, 8);
+        s.ctl->tail = tail0 + freed;
+    }
+}
+
 // compaction of the freed blocks by one CTA (all threads of the CTA must call it)
 __device__ __forceinline__ void evict_push_phase(const Geom &g, const DevState &s, const int *ctx, const int *ent_off,
                                                  int n, int total, unsigned long long stamp) {
     const unsigned long long tail0 = s.ctl->tail;
     int carry = 0;
-    for (int base = 0; base < total; base += PLAN_THREADS * EVICT_ITEMS) {
-        const int e0 = base + threadIdx.x * EVICT_ITEMS;
+    for (int base = 0; base < total; base += EVICT_TILE) {
         int blk[EVICT_ITEMS];
-        // locate the first entry once, then walk (context, position) forward: all table reads are independent
-        int ci = e0 < total ? find_ctx_index(ent_off, n, e0) : 0;
-#pragma unroll
-        for (int k = 0; k < EVICT_ITEMS; ++k) {
-            const int e = e0 + k;
-            blk[k] = -1;
-            if (e < total) {
-                while (e >= ent_off[ci + 1]) ++ci;
-                blk[k] = s.tables[(long long)ctx[ci] * g.max_blk + (e - ent_off[ci])];
-            }
-        }
-        int rc[EVICT_ITEMS];
-        unsigned long long lp[EVICT_ITEMS];
-#pragma unroll
-        for (int k = 0; k < EVICT_ITEMS; ++k) {
-            rc[k] = blk[k] >= 0 ? s.refcount[blk[k]] : 1;
-            lp[k] = blk[k] >= 0 ? s.last_pos[blk[k]] : 0ull;
-        }
-        int cnt = 0;
-        unsigned flags = 0;
-#pragma unroll
-        for (int k = 0; k < EVICT_ITEMS; ++k) {
-            const bool f = blk[k] >= 0 && rc[k] == 0 && lp[k] == (stamp | (unsigned long long)(unsigned)(e0 + k));
-            flags |= (f ? 1u : 0u) << k;
-            cnt += f;
-        }
+        const unsigned flags =
+            evict_thread_flags(g, s, ctx, ent_off, n, total, base + threadIdx.x * EVICT_ITEMS, stamp, blk);
         int tot;
-        int pos = carry + block_exclusive_scan(cnt, &tot);
-#pragma unroll
-        for (int k = 0; k < EVICT_ITEMS; ++k)
-            if (flags & (1u << k)) {
-                s.ring[(tail0 + (unsigned long long)pos) % (unsigned long long)g.NB] = blk[k];
-                ++pos;
-            }
+        const int pos = carry + block_exclusive_scan(__popc(flags), &tot);
+        evict_write_ring(g, s, tail0, pos, flags, blk);
         carry += tot;
     }
-    if (s.cat_len)
-        for (int i = threadIdx.x; i < n; i += blockDim.x) s.cat_len[ctx[i]] = -1;
-    if (threadIdx.x == 0) {
-        if (tail0 + carry - s.ctl->head > (unsigned long long)g.NB) set_status(s.ctl, AAF_ERR_CORRUPT, 8);
-        s.ctl->tail = tail0 + carry;
+    evict_finish(g, s, ctx, n, tail0, carry);
+}
+
+// Large batches: the same compaction over a grid, one tile of EVICT_TILE entries per CTA.
+//   count   : freed blocks per tile
+//   scan    : exclusive prefix sum of the tile counts (one CTA), ring tail and catalog update
+//   scatter : every tile recomputes its flags and writes its ids at tail0 + tile offset + local rank
+__global__ void __launch_bounds__(PLAN_THREADS) evict_count_kernel(Geom g, DevState s,
+                                                                   const EvictArgs *__restrict__ a, int n, int total,
+                                                                   unsigned long long stamp, int *tile_count) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    int blk[EVICT_ITEMS];
+    const unsigned flags = evict_thread_flags(g, s, ctx, ctx + n, n, total,
+                                              blockIdx.x * EVICT_TILE + threadIdx.x * EVICT_ITEMS, stamp, blk);
+    int tot;
+    block_exclusive_scan(__popc(flags), &tot);
+    if (threadIdx.x == 0) tile_count[blockIdx.x] = tot;
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) evict_scan_kernel(Geom g, DevState s,
+                                                                  const EvictArgs *__restrict__ a, int n, int n_tiles,
+                                                                  int *tile_count) {
+    const int *ctx = reinterpret_cast<const int *>(a + 1);
+    const unsigned long long tail0 = s.ctl->tail;
+    int carry = 0;
+    for (int base = 0; base < n_tiles; base += blockDim.x) {
+        const int t = base + threadIdx.x;
+        const int v = t < n_tiles ? tile_count[t] : 0;
+        int tot;
+        const int ex = block_exclusive_scan(v, &tot);
+        if (t < n_tiles) tile_count[t] = carry + ex;  // in place: count -> offset
+        carry += tot;
     }
+    if (threadIdx.x == 0) s.ctl->evict_tail0 = tail0;  // the scatter kernel needs the tail before this call
+    evict_finish(g, s, ctx, n, tail0, carry);
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) evict_scatter_kernel(Geom g, DevState s,
+                                                                     const EvictArgs *__restrict__ a, int n,
+                                                                     int total, unsigned long long stamp,
+                                                                     const int *tile_off) {
+    __shared__ int sh_args[EVICT_STAGE];
+    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    int blk[EVICT_ITEMS];
+    const unsigned flags = evict_thread_flags(g, s, ctx, ctx + n, n, total,
+                                              blockIdx.x * EVICT_TILE + threadIdx.x * EVICT_ITEMS, stamp, blk);
+    int tot;
+    const int pos = tile_off[blockIdx.x] + block_exclusive_scan(__popc(flags), &tot);
+    evict_write_ring(g, s, s.ctl->evict_tail0, pos, flags, blk);
 }
 
 __global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, const EvictArgs *__restrict__ a,
@@ -512,14 +581,6 @@ __global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, 
     const int *ent_off = ctx + n;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x)
         evict_release_entry(g, s, ctx, ent_off, n, e, stamp);
-}
-
-__global__ void __launch_bounds__(PLAN_THREADS) evict_push_kernel(Geom g, DevState s,
-                                                                  const EvictArgs *__restrict__ a, int n, int total,
-                                                                  unsigned long long stamp) {
-    __shared__ int sh_args[EVICT_STAGE];
-    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
-    evict_push_phase(g, s, ctx, ctx + n, n, total, stamp);
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS) evict_fused_kernel(Geom g, DevState s,
@@ -732,11 +793,12 @@ cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args
         evict_fused_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp);
         return cudaGetLastError();
     }
-    *n_launches = 2;
+    *n_launches = 4;
+    const int n_tiles = (total + EVICT_TILE - 1) / EVICT_TILE;
     evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev, n, total, stamp);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    evict_push_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp);
+    evict_count_kernel<<<n_tiles, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp, s.tile_count);
+    evict_scan_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, n_tiles, s.tile_count);
+    evict_scatter_kernel<<<n_tiles, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp, s.tile_count);
     return cudaGetLastError();
 }
 

@@ -27,7 +27,7 @@ namespace {
 constexpr int ARG_SLOTS = 16;
 
 struct Layout {
-    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, cat_origin, cat_parent, cat_born, cat_parent_born, total;
+    size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, cat_origin, cat_parent, cat_born, cat_parent_born, tile_count, total;
     int max_pieces, max_batch;
 };
 
@@ -64,6 +64,8 @@ Layout make_layout(const aaf_kv_pool_desc *d) {
     L.cat_parent = off; off = align_up(off + sizeof(int) * (size_t)d->max_ctx, 256);
     L.cat_born = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
     L.cat_parent_born = off; off = align_up(off + sizeof(long long) * (size_t)d->max_ctx, 256);
+    L.tile_count = off;
+    off = align_up(off + sizeof(int) * ((size_t)d->max_ctx * d->max_blocks_per_ctx / 8192 + 2), 256);
     L.total = off;
     return L;
 }
@@ -408,6 +410,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
     p->s.cat_parent = reinterpret_cast<int *>(ws + lay.cat_parent);
     p->s.cat_born = reinterpret_cast<long long *>(ws + lay.cat_born);
     p->s.cat_parent_born = reinterpret_cast<long long *>(ws + lay.cat_parent_born);
+    p->s.tile_count = reinterpret_cast<int *>(ws + lay.tile_count);
     p->len.assign((size_t)desc->max_ctx, -1);
     p->free_lb = desc->n_blocks;
 
