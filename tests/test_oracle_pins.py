@@ -89,11 +89,72 @@ def test_worked_example_w1():
                         assert got == bytes(row), "a never-written slot must keep its initial bytes"
                     else:
                         assert got == token_row(names[tok], l, kv, row)
+    assert o.stats()["rows_copied"] == int(g["rows_copied"])
     st, _ = o.evict([P, c2])
     assert st == 0
     assert o.refcounts().tolist() == [int(x) for x in g["refcount"].split()]
     assert o.free_list().tolist() == [int(x) for x in g["free_list"].split()]
     check_conservation(snapshot(o), NB, BS)
+
+
+def _w2_state():
+    """Steps 1-5 of the second worked example; returns (oracle, golden values, handles)."""
+    g = _read_kv(os.path.join(GOLD, "worked_example_w2.txt"))
+    NB, BS = int(g["NB"]), int(g["BS"])
+    L, row = 2, 8
+    o = paged.PagedOracle(L, 1, 4, BS, 2, NB, 6, 8, [int(x) for x in g["ring"].split()])
+    names = {f"a{i}": i for i in range(8)}
+    names.update({f"c{i}": 50 + i for i in range(5)})
+    names["y0"] = 90
+    enc = lambda toks: encode_tokens([names[t] for t in toks], L, row)
+    ints = lambda key: [int(x) for x in g[key].split()]
+
+    st, A = o.imp(enc([f"a{i}" for i in range(8)]), 8)
+    assert (st, A) == (0, 0) and o.table(A).tolist() == ints("A.table")
+    st, B = o.compose([A, A])
+    assert (st, B) == (0, 1) and o.table(B).tolist() == ints("B.table")
+    assert o.refcounts().tolist() == ints("refcount.after_compose")
+    st, Cc = o.imp(enc([f"c{i}" for i in range(5)]), 5)
+    assert (st, Cc) == (0, 2) and o.table(Cc).tolist() == ints("C.table")
+    st, (D,) = o.fork(Cc, 1)
+    assert (st, D) == (0, 3)
+    assert o.append([D], [1], [enc(["y0"])])[0] == 0
+    assert o.table(D).tolist() == ints("D.table")
+    pv = o.pool_view()
+    for s, tok in enumerate(g["block3"].split()):
+        for l in range(L):
+            for kv in range(2):
+                want = bytes(row) if tok == "." else token_row(names[tok], l, kv, row)
+                assert bytes(pv[l, 3, kv, s]) == want
+    assert o.refcounts().tolist() == ints("refcount.before_evict")
+    assert o.stats()["rows_copied"] == int(g["rows_copied.before_evict"])
+    return o, g, (A, B, Cc, D)
+
+
+def test_worked_example_w2_order_of_blocks_freed_by_one_evict():
+    """Pins the push order of a batched evict: flattened (context, table position) order, a block
+    pushed at its last occurrence -- with a block named twice by one victim and once more by another."""
+    o, g, (A, B, Cc, D) = _w2_state()
+    ints = lambda key: [int(x) for x in g[key].split()]
+    assert o.evict([B, D, A])[0] == 0
+    assert o.refcounts().tolist() == ints("refcount.after_evict")
+    assert o.free_list().tolist() == ints("free_list.after_evict")
+    assert o.live_ctxs() == ints("live.after_evict")
+    check_conservation(snapshot(o), o.NB, o.BS)
+
+
+def test_worked_example_w2_order_of_blocks_freed_by_scored_eviction():
+    """The same pin for the scored eviction loop: victims oldest first, each victim's blocks released
+    front to back, shared blocks survive until their last holder goes."""
+    o, g, (A, B, Cc, D) = _w2_state()
+    ints = lambda key: [int(x) for x in g[key].split()]
+    assert o.materialize(A, 0, 8)[0] == 0
+    st, victims = o.evict_to_budget(0.0, 0.0, 1.0, 3)
+    assert st == 0 and victims == ints("budget.victims")
+    assert o.refcounts().tolist() == ints("budget.refcount")
+    assert o.free_list().tolist() == ints("budget.free_list")
+    assert o.live_ctxs() == [A]
+    check_conservation(snapshot(o), o.NB, o.BS)
 
 
 # ---------------------------------------------------------------- P1 / P2: transfer preserves content
