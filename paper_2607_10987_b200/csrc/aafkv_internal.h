@@ -7,17 +7,22 @@
 
 namespace aafkv {
 
-// One contiguous copy, described once for all (layer, K/V) planes:
-//   plane (l, kv):  src + l * src_sl + kv * src_skv  ->  dst + l * dst_sl + kv * dst_skv,  nbytes bytes.
-// For a pool operand the strides are (layer_stride, run); for an n-token transfer buffer they are
-// (2 * n * row, n * row).  nbytes is a multiple of row (hence of 16); 0 marks an unused slot.
+// One copy, described once for all (layer, K/V) planes:
+//   plane (l, kv):  src + l * src_sl + kv * src_skv  ->  dst + l * dst_sl + kv * dst_skv,  nbytes bytes,
+// optionally followed by a second part from the same operand: nbytes2 bytes from src + src2_off (same
+// plane strides) that land directly behind the first part, at dst + nbytes.  The second part lets a
+// destination block that is filled from two source blocks (the shifted copy of a compose) be one unit of
+// work with one contiguous store.  For a pool operand the strides are (layer_stride, run); for an
+// n-token transfer buffer they are (2 * n * row, n * row).  nbytes and nbytes2 are multiples of row
+// (hence of 16) and nbytes + nbytes2 <= run; nbytes == 0 marks an unused slot.
 struct __align__(16) Piece {
     const char *src;
     char *dst;
     long long src_sl, src_skv;
     long long dst_sl, dst_skv;
     unsigned int nbytes;
-    unsigned int pad[3];
+    unsigned int nbytes2;
+    long long src2_off;
 };
 static_assert(sizeof(Piece) == 64, "Piece must be 64 bytes");
 
@@ -34,7 +39,12 @@ struct DevCtl {
     unsigned int one;                  // constant 1: source of the host-visible chunk completion flags
     unsigned int pad32;
     unsigned long long evict_tail0;    // ring tail before the current large evict (read by its scatter kernel)
-    unsigned long long pad[7];
+    // work distribution of the copy engines: CTAs draw unit tickets from copy_ticket; the last CTA to leave
+    // (counted in copy_done) sets both back to 0, so every launch starts from 0 without a host-side reset
+    unsigned long long copy_ticket;
+    unsigned int copy_done;
+    unsigned int pad32b;
+    unsigned long long pad[5];
 };
 static_assert(sizeof(DevCtl) == 128, "DevCtl layout");
 

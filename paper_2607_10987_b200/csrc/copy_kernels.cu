@@ -6,6 +6,13 @@
 // the bound is HBM bandwidth: what matters is enough independent 16-byte accesses in flight per
 // SM, fully coalesced, and a persistent grid of exactly one resident wave (a multiple of the SM count).
 //
+// Work distribution: the SMs of a B200 do not get equal shares of the memory bandwidth (measured: with
+// equal static shares some CTAs were done after 70 % of the kernel's time and the slowest set the
+// pace), so the BULK and WARP engines hand units out dynamically: a CTA (a warp) draws the next unit
+// (group of 32 units) from a ticket counter in the pool's control block.  The last CTA to leave sets
+// the counter back to 0.  Launches that share a control block must therefore not overlap on the GPU;
+// the library issues all copy launches of a pool to the caller's stream, in order.
+//
 //   BULK : one elected thread per CTA drives a ring of shared-memory stages with
 //          cp.async.bulk (global -> shared, completion on an mbarrier) and
 //          cp.async.bulk (shared -> global, bulk async-group); no registers touch the data and the
@@ -14,7 +21,7 @@
 //   WARP : 16-byte streaming loads/stores scheduled per warp, 32 units decoded at once; the default
 //          for small and ragged pieces.
 //   VEC  : 256 threads per CTA, each thread keeps UNROLL 16-byte streaming loads in flight and
-//          then stores them; one chunk per CTA iteration.  Kept as the plain baseline.
+//          then stores them; one chunk per CTA iteration, equal static shares.  Kept as the plain baseline.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -27,9 +34,11 @@ namespace aafkv {
 // unit decomposition shared by all engines: unit u -> (chunk c, piece p, plane q), plane-major
 // so that neighbouring CTAs stream neighbouring addresses of the dense side.
 struct Unit {
-    const char *src;
+    const char *src;   // first part
+    const char *src2;  // second part (lands at dst + nbytes)
     char *dst;
-    unsigned nbytes;  // 0 = nothing to do
+    unsigned nbytes;   // bytes of the first part in this chunk
+    unsigned nbytes2;  // bytes of the second part in this chunk; nbytes + nbytes2 == 0: nothing to do
 };
 
 __device__ __forceinline__ Unit decode_unit(const Piece *__restrict__ pieces, long long u, int n_slots, int plane0,
@@ -47,15 +56,38 @@ __device__ __forceinline__ Unit decode_unit(const Piece *__restrict__ pieces, lo
     reinterpret_cast<uint4 *>(&pc)[3] = w3;
     Unit r;
     const unsigned off = (unsigned)c * chunk;
-    if (off >= pc.nbytes) {
-        r.src = nullptr; r.dst = nullptr; r.nbytes = 0;
+    const unsigned tot = pc.nbytes ? pc.nbytes + pc.nbytes2 : 0u;  // nbytes == 0: unused slot, whatever else it holds
+    if (off >= tot) {
+        r.src = nullptr; r.src2 = nullptr; r.dst = nullptr; r.nbytes = 0; r.nbytes2 = 0;
         return r;
     }
     const long long l = q >> 1, kv = q & 1;
-    r.src = pc.src + l * pc.src_sl + kv * pc.src_skv + off;
+    const char *base = pc.src + l * pc.src_sl + kv * pc.src_skv;
+    const unsigned len = min(chunk, tot - off);
+    const unsigned na = off < pc.nbytes ? min(len, pc.nbytes - off) : 0u;  // share of the first part
+    r.src = base + off;
+    r.src2 = base + pc.src2_off + (off + na - pc.nbytes);
     r.dst = pc.dst + l * pc.dst_sl + kv * pc.dst_skv + off;
-    r.nbytes = min(chunk, pc.nbytes - off);
+    r.nbytes = na;
+    r.nbytes2 = len - na;
     return r;
+}
+
+// Ticket counter of the dynamic work distribution (see the header comment).
+__device__ __forceinline__ long long take_ticket(DevCtl *ctl) { return (long long)atomicAdd(&ctl->copy_ticket, 1ull); }
+// Called once per CTA when it has drawn its last ticket: the last CTA of the grid re-arms the counters.
+__device__ __forceinline__ void leave_copy(DevCtl *ctl) {
+    __threadfence();
+    if (atomicAdd(&ctl->copy_done, 1u) == gridDim.x - 1) {
+        ctl->copy_ticket = 0;
+        ctl->copy_done = 0;
+        __threadfence();
+    }
+}
+
+// 16-byte vector i of a unit: the first part's vectors, then the second part's
+__device__ __forceinline__ const uint4 *unit_vec(const uint4 *s4, const uint4 *s4b, unsigned nvec_a, unsigned i) {
+    return i < nvec_a ? s4 + i : s4b + (i - nvec_a);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -69,15 +101,16 @@ __global__ void __launch_bounds__(VEC_THREADS) copy_vec_kernel(const Piece *__re
     const long long total = (long long)n_slots * n_planes * cpp;
     for (long long u = blockIdx.x; u < total; u += gridDim.x) {
         const Unit un = decode_unit(pieces, u, n_slots, plane0, cpp, CHUNK);
-        if (un.nbytes == 0) continue;
+        if (un.nbytes + un.nbytes2 == 0) continue;
         const uint4 *__restrict__ s4 = reinterpret_cast<const uint4 *>(un.src);
+        const uint4 *__restrict__ s4b = reinterpret_cast<const uint4 *>(un.src2);
         uint4 *__restrict__ d4 = reinterpret_cast<uint4 *>(un.dst);
-        const unsigned nvec = un.nbytes >> 4;
+        const unsigned nvec_a = un.nbytes >> 4, nvec = (un.nbytes + un.nbytes2) >> 4;
         uint4 v[UNROLL];
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) {
             const unsigned i = threadIdx.x + k * VEC_THREADS;
-            if (i < nvec) v[k] = __ldcs(s4 + i);
+            if (i < nvec) v[k] = __ldcs(unit_vec(s4, s4b, nvec_a, i));
         }
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) {
@@ -96,31 +129,37 @@ __global__ void __launch_bounds__(VEC_THREADS) copy_vec_kernel(const Piece *__re
 // latency; full runs are split into 32*U*16-byte chunks handled by neighbouring warps.
 template <int UNROLL>
 __global__ void __launch_bounds__(VEC_THREADS) copy_warp_kernel(const Piece *__restrict__ pieces, int n_slots,
-                                                                int plane0, int n_planes, int cpp) {
+                                                                int plane0, int n_planes, int cpp, DevCtl *ctl) {
     constexpr unsigned CHUNK = 32 * UNROLL * 16;
     constexpr unsigned FULL = 0xffffffffu;
     const long long total = (long long)n_slots * n_planes * cpp;
+    const long long groups = (total + 31) / 32;  // a ticket is worth 32 consecutive units
     const int lane = threadIdx.x & 31;
-    const long long warps = (long long)gridDim.x * (VEC_THREADS / 32);
-    const long long gw = (long long)blockIdx.x * (VEC_THREADS / 32) + (threadIdx.x >> 5);
-    for (long long base = gw * 32; base < total; base += warps * 32) {
+    long long grp = lane == 0 ? take_ticket(ctl) : 0;
+    grp = __shfl_sync(FULL, grp, 0);
+    while (grp < groups) {
+        long long grp_next = lane == 0 ? take_ticket(ctl) : 0;  // drawn early: its latency hides behind the copies
+        const long long base = grp * 32;
         Unit mine;
-        mine.src = nullptr; mine.dst = nullptr; mine.nbytes = 0;
+        mine.src = nullptr; mine.src2 = nullptr; mine.dst = nullptr; mine.nbytes = 0; mine.nbytes2 = 0;
         if (base + lane < total) mine = decode_unit(pieces, base + lane, n_slots, plane0, cpp, CHUNK);
-        unsigned todo = __ballot_sync(FULL, mine.nbytes != 0);
+        unsigned todo = __ballot_sync(FULL, mine.nbytes + mine.nbytes2 != 0);
         while (todo) {
             const int j = __ffs(todo) - 1;
             todo &= todo - 1;
             const uint4 *__restrict__ s4 = reinterpret_cast<const uint4 *>(
                 __shfl_sync(FULL, reinterpret_cast<unsigned long long>(mine.src), j));
+            const uint4 *__restrict__ s4b = reinterpret_cast<const uint4 *>(
+                __shfl_sync(FULL, reinterpret_cast<unsigned long long>(mine.src2), j));
             uint4 *__restrict__ d4 =
                 reinterpret_cast<uint4 *>(__shfl_sync(FULL, reinterpret_cast<unsigned long long>(mine.dst), j));
-            const unsigned nvec = __shfl_sync(FULL, mine.nbytes, j) >> 4;
+            const unsigned nvec_a = __shfl_sync(FULL, mine.nbytes, j) >> 4;
+            const unsigned nvec = nvec_a + (__shfl_sync(FULL, mine.nbytes2, j) >> 4);
             uint4 v[UNROLL];
 #pragma unroll
             for (int k = 0; k < UNROLL; ++k) {
                 const unsigned i = lane + k * 32;
-                if (i < nvec) v[k] = __ldcs(s4 + i);
+                if (i < nvec) v[k] = __ldcs(unit_vec(s4, s4b, nvec_a, i));
             }
 #pragma unroll
             for (int k = 0; k < UNROLL; ++k) {
@@ -128,7 +167,10 @@ __global__ void __launch_bounds__(VEC_THREADS) copy_warp_kernel(const Piece *__r
                 if (i < nvec) __stcs(d4 + i, v[k]);
             }
         }
+        grp = __shfl_sync(FULL, grp_next, 0);
     }
+    __syncthreads();  // every warp of the CTA has drawn its last ticket
+    if (threadIdx.x == 0) leave_copy(ctl);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -220,6 +262,8 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
                                                        int l2_hints, DevCtl *ctl) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long bars[BULK_MAX_STAGES];
+    __shared__ char *dstq[BULK_MAX_STAGES];   // destination and size of the unit held by each stage
+    __shared__ unsigned nbq[BULK_MAX_STAGES];  // (indexed dynamically: shared memory, not a local frame)
     if (threadIdx.x != 0) return;
 
     const long long total = (long long)n_slots * n_planes * cpp;
@@ -230,25 +274,27 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
-    char *dstq[BULK_MAX_STAGES];
-    unsigned nbq[BULK_MAX_STAGES];
-    long long u_next = blockIdx.x;  // next unit to look at for loading
-    int k_load = 0;                 // units whose load has been issued
-    int k_store = 0;                // units whose store has been issued
+    long long u_next = take_ticket(ctl);  // next unit to look at for loading
+    int k_load = 0;                       // units whose load has been issued
+    int k_store = 0;                      // units whose store has been issued
     bool timed_out = false;
 
-    // finds the next non-empty unit and issues its load into stage k_load % stages
+    // finds the next non-empty unit and issues its load (two loads for a two-part unit) into stage
+    // k_load % stages; the ticket after it is drawn at once, so that its latency hides behind the copies
     auto issue_load = [&]() -> bool {
         while (u_next < total) {
             const Unit un = decode_unit(pieces, u_next, n_slots, plane0, cpp, chunk);
-            u_next += gridDim.x;
-            if (un.nbytes == 0) continue;
+            u_next = take_ticket(ctl);
+            const unsigned nb = un.nbytes + un.nbytes2;
+            if (nb == 0) continue;
             const int s = k_load % stages;
             const unsigned bar = smem_u32(&bars[s]);
-            mbar_expect_tx(bar, un.nbytes);
-            bulk_g2s(smem0 + (unsigned)s * chunk, un.src, un.nbytes, bar, pol, hint_ld);
+            const unsigned stage = smem0 + (unsigned)s * chunk;
+            mbar_expect_tx(bar, nb);
+            if (un.nbytes) bulk_g2s(stage, un.src, un.nbytes, bar, pol, hint_ld);
+            if (un.nbytes2) bulk_g2s(stage + un.nbytes, un.src2, un.nbytes2, bar, pol, hint_ld);
             dstq[s] = un.dst;
-            nbq[s] = un.nbytes;
+            nbq[s] = nb;
             ++k_load;
             return true;
         }
@@ -279,6 +325,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
             mbar_wait_bounded(smem_u32(&bars[k % stages]), (unsigned)(k / stages) & 1u);
     }
     bulk_wait_all();
+    leave_copy(ctl);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -360,7 +407,7 @@ static void launch_warp(const CopyTuning &t, const DevState &s, int n_slots, int
     const long long need = (total + 255) / 256;  // CTAs needed if every warp takes one round of 32 units
     const long long cap = (long long)sm_count * t.warp_ctas;
     const int grid = (int)(need < cap ? (need < 1 ? 1 : need) : cap);
-    copy_warp_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp);
+    copy_warp_kernel<UNROLL><<<grid, VEC_THREADS, 0, st>>>(s.pieces, n_slots, plane0, n_planes, cpp, s.ctl);
 }
 
 // AUTO: pieces of about a run or more -> the bulk engine (fastest, and it leaves the SMs idle);

@@ -35,8 +35,14 @@ __device__ __forceinline__ Piece make_piece(const char *src, long long ssl, long
     p.src_sl = ssl; p.src_skv = sskv;
     p.dst_sl = dsl; p.dst_skv = dskv;
     p.nbytes = nbytes;
-    p.pad[0] = p.pad[1] = p.pad[2] = 0;
+    p.nbytes2 = 0;
+    p.src2_off = 0;
     return p;
+}
+// marks a piece slot unused (both parts: a slot may still hold an earlier operator's two-part piece)
+__device__ __forceinline__ void clear_piece(Piece &p) {
+    p.nbytes = 0;
+    p.nbytes2 = 0;
 }
 __device__ __forceinline__ char *pool_slot(const Geom &g, int b, long long slot) {
     return g.pool + (long long)b * 2 * g.run + slot * g.row;
@@ -129,6 +135,11 @@ __global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState 
     for (long long j = j0 + blockIdx.x * blockDim.x + threadIdx.x; j <= j1; j += (long long)gridDim.x * blockDim.x) {
         const long long lo = max(t0, j * g.BS), hi = min(t1, (j + 1) * g.BS);
         const int b = table[j];
+        if (b < 0 || b >= g.NB) {  // never gather through an entry that does not name a pool block
+            clear_piece(s.pieces[j - j0]);
+            set_status(s.ctl, AAF_ERR_CORRUPT, 10);
+            continue;
+        }
         s.pieces[j - j0] = make_piece(pool_slot(g, b, lo - j * g.BS), g.layer_stride, g.run, dst + (lo - t0) * g.row,
                                       2 * n * g.row, n * g.row, (unsigned)((hi - lo) * g.row));
     }
@@ -151,7 +162,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevSt
     int *table = s.tables + (long long)ctx * g.max_blk;
     for (int j = threadIdx.x; j < nblk; j += blockDim.x) {
         if (!ok) {
-            s.pieces[j].nbytes = 0;
+            clear_piece(s.pieces[j]);
             continue;
         }
         const int b = ring_at(s.ring, head0 + j, g.NB);
@@ -266,7 +277,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
     unsigned long long my_bytes = 0;
     for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) {
         if (!ok) {
-            s.pieces[sl].nbytes = 0;
+            clear_piece(s.pieces[sl]);
             continue;
         }
         int lo = 0, hi = n - 1;  // last entry whose piece_off <= sl
@@ -295,7 +306,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
                 atomicAdd(&s.ctl->cow_count, 1ull);
                 my_bytes += (unsigned long long)(r * g.row * 2 * g.L);
             } else {
-                s.pieces[sl].nbytes = 0;
+                clear_piece(s.pieces[sl]);
             }
             continue;
         }
@@ -338,7 +349,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 //                   reference if it ends the result, else re-packed into a fresh block through the
 //                   segment's single piece slot)
 //   copy segment  : item w -> destination block nblk(off)-(off%BS>0) + w, which receives tokens
-//                   from at most two source blocks (two piece slots per item)
+//                   from at most two source blocks (one two-part piece per item)
 __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
                                                                     const ComposeSeg *__restrict__ segs_host, int m,
                                                                     int total_work, int total_fresh, int total_slots,
@@ -349,7 +360,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
     const bool ok = (tail - head0) >= (unsigned long long)total_fresh;
     int *out = s.tables + (long long)out_ctx * g.max_blk;
     if (!ok) {
-        for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) s.pieces[sl].nbytes = 0;
+        for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) clear_piece(s.pieces[sl]);
     }
     unsigned long long my_bytes = 0;
     for (int it = threadIdx.x; ok && it < total_work; it += blockDim.x) {
@@ -389,17 +400,16 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
             const long long s_lo = lo_t - sg.off, s_hi = hi_t - sg.off;  // source token range
             const long long sb0 = s_lo / g.BS;
             const long long a_hi = min(s_hi, (sb0 + 1) * g.BS);
-            Piece *pp = s.pieces + sg.piece_off + 2 * w;
-            pp[0] = make_piece(pool_slot(g, st[sb0], s_lo - sb0 * g.BS), g.layer_stride, g.run,
-                               pool_slot(g, db, lo_t - d * g.BS), g.layer_stride, g.run,
-                               (unsigned)((a_hi - s_lo) * g.row));
+            // one two-part piece per destination block: the rows from source block sb0, then (if the range
+            // crosses into it) the rows from the start of source block sb0 + 1, stored as one contiguous run
+            Piece pc = make_piece(pool_slot(g, st[sb0], s_lo - sb0 * g.BS), g.layer_stride, g.run,
+                                  pool_slot(g, db, lo_t - d * g.BS), g.layer_stride, g.run,
+                                  (unsigned)((a_hi - s_lo) * g.row));
             if (a_hi < s_hi) {
-                pp[1] = make_piece(pool_slot(g, st[sb0 + 1], 0), g.layer_stride, g.run,
-                                   pool_slot(g, db, lo_t - d * g.BS + (a_hi - s_lo)), g.layer_stride, g.run,
-                                   (unsigned)((s_hi - a_hi) * g.row));
-            } else {
-                pp[1].nbytes = 0;
+                pc.nbytes2 = (unsigned)((s_hi - a_hi) * g.row);
+                pc.src2_off = pool_slot(g, st[sb0 + 1], 0) - pc.src;
             }
+            s.pieces[sg.piece_off + w] = pc;
             my_bytes += (unsigned long long)((s_hi - s_lo) * g.row * 2 * g.L);
         }
     }

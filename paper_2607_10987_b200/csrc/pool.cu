@@ -751,7 +751,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
             r.mode = 1;
             const long long items = (off + T - 1) / BS - off / BS + 1;
             work += items;
-            slots += 2 * items;
+            slots += items;  // one two-part piece per destination block
             copied_tokens += T;
             fresh += nblk_of(p, off + T) - nblk_of(p, off);
         }
