@@ -206,7 +206,7 @@ def extra_report(args):
     import torch
 
     from paper_2607_10987_b200 import binding
-    from paper_2607_10987_b200.replay_backend import GpuBackend
+    from tests.gpu_backend import GpuBackend
     from workloads import churn
     from workloads.replay import replay
 

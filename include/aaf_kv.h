@@ -46,9 +46,13 @@
  *
  * Errors: every call returns 0 (AAF_OK) or a negative aaf_status.  Everything the host
  * can know is checked before anything is launched, so an error return means no state
- * changed.  Conditions only the device can see (a corrupted ring or reference count, a
- * bounded wait that gave up) never trap: they set a sticky status word that
- * aaf_kv_sync_status returns and clears.
+ * changed -- with one exception: AAF_ERR_CUDA from an operator means that a CUDA runtime
+ * call failed, possibly after a metadata kernel had already been enqueued, so the host's
+ * view of the pool can no longer be trusted.  The pool is then unusable: every later
+ * operator call on it returns AAF_ERR_CUDA, and the only useful call left is
+ * aaf_kv_pool_destroy.  Conditions only the device can see (a corrupted ring or
+ * reference count, a bounded wait that gave up) never trap: they set a sticky status
+ * word that aaf_kv_sync_status returns and clears.
  */
 #ifndef AAF_KV_H
 #define AAF_KV_H
@@ -314,9 +318,12 @@ int aaf_kv_set_timing(aaf_kv_pool *pool, int enable);       /* bracket copy kern
  *   - All calls on a device share the one array, which keeps the previous call's contents; each
  *     call clears or overwrites what it reads.  Two calls that overlap on the GPU (different
  *     streams, or host threads racing) corrupt each other: keep them on one stream or order them.
- *   - pool_base_dev, dst_dev: device, 16-byte aligned; block_table_host: host, read before return.
- * Errors: INVALID_ARG (pointers, geometry, range, a table entry outside [0, n_blocks)),
- * DST_TOO_SMALL, SCRATCH_LIMIT, CUDA. */
+ *   - pool_base_dev, dst_dev: memory of the current device, 16-byte aligned.  block_table_host: host
+ *     memory; its entries are checked before the call returns and uploaded by an asynchronous copy on
+ *     `stream`, so the array must stay unchanged until the stream has run the call (a pageable array
+ *     happens to be read before return; a pinned one is not).
+ * Errors: INVALID_ARG (pointers, memory of another device, geometry, range, a table entry outside
+ * [0, n_blocks)), DST_TOO_SMALL, SCRATCH_LIMIT, CUDA. */
 #define AAF_NOALLOC_MAX_BLOCKS 4096
 int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t layer_stride_bytes, int32_t n_layers,
                                int32_t n_kv_heads, int32_t head_dim, int32_t block_size, int32_t elt_bytes,

@@ -106,7 +106,7 @@ struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
 // `clock` is the logical clock of the call (count of successful state-touching calls); planners stamp
 // it into the catalog.  A DevState without catalog arrays (cat_len == nullptr) skips the stamping.
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
-                                    long long clock, cudaStream_t st);
+                                    long long clock, cudaStream_t st, int table_j0 = 0);
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
                                long long clock, cudaStream_t st);
 cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,

@@ -127,14 +127,17 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *total) {
 
 // ------------------------------------------------------------------------------------------
 // materialize: one piece per block of the token range
+// `table_j0`: table position held by the first entry of the context's table row (0 for a pool; a caller that
+// uploads only the slice of a table it needs passes the slice's first position)
 __global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState s, int ctx, long long t0,
-                                                               long long t1, char *dst, long long clock) {
+                                                               long long t1, char *dst, long long clock,
+                                                               int table_j0) {
     const long long j0 = t0 / g.BS, j1 = (t1 - 1) / g.BS;
     const long long n = t1 - t0;
     const int *table = s.tables + (long long)ctx * g.max_blk;
     for (long long j = j0 + blockIdx.x * blockDim.x + threadIdx.x; j <= j1; j += (long long)gridDim.x * blockDim.x) {
         const long long lo = max(t0, j * g.BS), hi = min(t1, (j + 1) * g.BS);
-        const int b = table[j];
+        const int b = table[j - table_j0];
         if (b < 0 || b >= g.NB) {  // never gather through an entry that does not name a pool block
             clear_piece(s.pieces[j - j0]);
             set_status(s.ctl, AAF_ERR_CORRUPT, 10);
@@ -768,9 +771,9 @@ static int grid_for(long long items, int threads, int cap) {
 }
 
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
-                                    long long clock, cudaStream_t st) {
+                                    long long clock, cudaStream_t st, int table_j0) {
     const long long nb = (t1 - 1) / g.BS - t0 / g.BS + 1;
-    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst, clock);
+    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst, clock, table_j0);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,

@@ -72,22 +72,40 @@ extern "C" int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t laye
     if (n_layers < 1 || n_kv_heads < 1 || head_dim < 1 || block_size < 1 || elt_bytes < 1 || n_blocks < 1 ||
         n_table_blocks < 1)
         return AAF_ERR_INVALID_ARG;
-    const long long row = (long long)n_kv_heads * head_dim * elt_bytes;
-    const long long run = row * block_size;
-    if (row % 16 != 0 || run > (1ll << 30)) return AAF_ERR_INVALID_ARG;
+    // sizes are bounded before anything is multiplied: a row and a run fit 2^30 bytes, the layer count 2^16
+    if (n_layers > 65536) return AAF_ERR_INVALID_ARG;
+    long long row = 0, run = 0;
+    if (__builtin_mul_overflow((long long)n_kv_heads, (long long)head_dim, &row) ||
+        __builtin_mul_overflow(row, (long long)elt_bytes, &row) || row > (1ll << 30) ||
+        __builtin_mul_overflow(row, (long long)block_size, &run) || run > (1ll << 30))
+        return AAF_ERR_INVALID_ARG;
+    if (row % 16 != 0) return AAF_ERR_INVALID_ARG;
     if (layer_stride_bytes % 16 != 0 || layer_stride_bytes < (size_t)(2 * run * n_blocks)) return AAF_ERR_INVALID_ARG;
     if (tok_begin < 0 || tok_begin >= tok_end || tok_end > (long long)n_table_blocks * block_size)
         return AAF_ERR_INVALID_ARG;
     const long long n = tok_end - tok_begin;
-    if ((unsigned long long)dst_bytes < (unsigned long long)(n * 2 * n_layers * row)) return AAF_ERR_DST_TOO_SMALL;
     const long long j0 = tok_begin / block_size, j1 = (tok_end - 1) / block_size;
     const long long nb = j1 - j0 + 1;
-    if (nb > AAF_NOALLOC_MAX_BLOCKS) return AAF_ERR_SCRATCH_LIMIT;
+    if (nb > AAF_NOALLOC_MAX_BLOCKS) return AAF_ERR_SCRATCH_LIMIT;  // also bounds n: n <= 4096 * block_size
+    // n <= 2^12 * block_size and block_size * row <= 2^30, so n * row <= 2^42; times 2 * n_layers <= 2^17: no overflow
+    if ((unsigned long long)dst_bytes < (unsigned long long)(n * row) * 2ull * (unsigned long long)n_layers)
+        return AAF_ERR_DST_TOO_SMALL;
     for (long long j = j0; j <= j1; ++j)
         if (block_table_host[j] < 0 || block_table_host[j] >= n_blocks) return AAF_ERR_INVALID_ARG;
 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return AAF_ERR_CUDA;
+    // both buffers must be memory of the current device: the scratch and the launch shapes used below are
+    // this device's (the query allocates nothing)
+    for (const void *q : {pool_base_dev, static_cast<const void *>(dst_dev)}) {
+        cudaPointerAttributes pa{};
+        if (cudaPointerGetAttributes(&pa, q) != cudaSuccess) {
+            cudaGetLastError();
+            return AAF_ERR_INVALID_ARG;
+        }
+        if ((pa.type == cudaMemoryTypeDevice || pa.type == cudaMemoryTypeManaged) && pa.device != dev)
+            return AAF_ERR_INVALID_ARG;
+    }
     const int rc = setup_device(dev);
     if (rc != AAF_OK) return rc;
     NoAllocScratch *sc = g_scratch_ptr[dev];
@@ -107,9 +125,10 @@ extern "C" int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t laye
     g.pool = static_cast<char *>(const_cast<void *>(pool_base_dev));
     DevState s{};
     s.ctl = &sc->ctl;
-    s.tables = sc->table - j0;  // the planner indexes the table by absolute block position
+    s.tables = sc->table;  // holds entries j0 .. j1 of the caller's table: the planner subtracts j0
     s.pieces = sc->pieces;
-    if (launch_plan_materialize(g, s, 0, tok_begin, tok_end, static_cast<char *>(dst_dev), 0, st) != cudaSuccess)
+    if (launch_plan_materialize(g, s, 0, tok_begin, tok_end, static_cast<char *>(dst_dev), 0, st, (int)j0) !=
+        cudaSuccess)
         return AAF_ERR_CUDA;
     if (launch_copy(AAF_ENGINE_VEC, g_tuning[dev], g, s, (int)nb, 0, 2 * n_layers, run, g_sm_count[dev], st) !=
         cudaSuccess)

@@ -94,6 +94,7 @@ struct aaf_kv_pool {
     DevState s;
     Layout lay;
     int device = 0, sm_count = 148;
+    bool broken = false;  // a CUDA call failed after device state had changed: every later call returns AAF_ERR_CUDA
     CopyTuning tuning{};
     std::vector<long long> len;  // tokens per handle, -1 = free
     int live_ctx = 0;
@@ -133,6 +134,12 @@ namespace {
 
 long long nblk_of(const aaf_kv_pool *p, long long tokens) { return (tokens + p->g.BS - 1) / p->g.BS; }
 bool is_live(const aaf_kv_pool *p, int c) { return c >= 0 && c < p->g.max_ctx && p->len[c] >= 0; }
+// A CUDA runtime call failed after a planner may already have changed the device's metadata: the host mirror
+// can no longer be trusted, so the pool refuses all further work.
+int broke(aaf_kv_pool *p) {
+    p->broken = true;
+    return AAF_ERR_CUDA;
+}
 bool aligned16(const void *q) { return q && (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
 long long bpt_of(const aaf_kv_pool *p) { return 2ll * p->g.L * p->g.row; }
 
@@ -248,7 +255,7 @@ int run_copy(aaf_kv_pool *p, const PlanSlot &ps, int cls, int n_slots, long long
         if (p->pending.size() > 4096) drain_timing(p);
     }
     p->copy_launches[cls] += 1;
-    return e == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
+    return e == cudaSuccess ? AAF_OK : broke(p);
 }
 
 void fill_desc(const aaf_kv_pool *p, aaf_kv_xfer_desc *d, long long pos_start, long long n) {
@@ -276,7 +283,7 @@ int materialize_impl(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, int64_t t1, void
     if (launch_plan_materialize(p->g, ps.view, ctx, t0, t1, static_cast<char *>(dst_dev), p->clock + 1,
                                 p->meta_stream) != cudaSuccess ||
         !end_plan(p, ps, st))
-        return AAF_ERR_CUDA;
+        return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     const int n_slots = (int)((t1 - 1) / p->g.BS - t0 / p->g.BS + 1);
@@ -302,13 +309,13 @@ int import_impl(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *des
     if (src_host) {
         if (cudaMemcpyAsync(const_cast<void *>(src_dev), src_host, (size_t)(n * bpt_of(p)), cudaMemcpyHostToDevice,
                             st) != cudaSuccess)
-            return AAF_ERR_CUDA;
+            return broke(p);
     }
     const PlanSlot ps = begin_plan(p);
     if (launch_plan_import(p->g, ps.view, c, n, static_cast<const char *>(src_dev), p->clock + 1, p->meta_stream) !=
             cudaSuccess ||
         !end_plan(p, ps, st))
-        return AAF_ERR_CUDA;
+        return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= nb;
@@ -478,6 +485,7 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
 int aaf_kv_materialize(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_dev,
                        size_t dst_bytes, aaf_kv_xfer_desc *out_desc, void *stream) {
     if (!p) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
     return materialize_impl(p, ctx, tok_begin, tok_end, dst_dev, dst_bytes, out_desc,
                             static_cast<cudaStream_t>(stream));
@@ -487,6 +495,7 @@ int aaf_kv_materialize_host(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, in
                             size_t dst_bytes, void *staging_dev, size_t staging_bytes, aaf_kv_xfer_desc *out_desc,
                             void *stream) {
     if (!p || !dst_host) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (is_live(p, ctx) && tok_begin >= 0 && tok_begin < tok_end &&
@@ -496,12 +505,13 @@ int aaf_kv_materialize_host(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, in
     if (rc != AAF_OK) return rc;
     const size_t bytes = (size_t)((tok_end - tok_begin) * bpt_of(p));
     return cudaMemcpyAsync(dst_host, staging_dev, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess ? AAF_OK
-                                                                                                   : AAF_ERR_CUDA;
+                                                                                                   : broke(p);
 }
 
 int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
                   void *stream) {
     if (!p) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
     return import_impl(p, src_dev, desc, out_ctx, static_cast<cudaStream_t>(stream), nullptr);
 }
@@ -509,6 +519,7 @@ int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *d
 int aaf_kv_import_host(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
                        size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream) {
     if (!p || !src_host || !desc) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
     if (desc->n_tokens >= 1 && (unsigned long long)staging_bytes < (unsigned long long)(desc->n_tokens * bpt_of(p)))
         return AAF_ERR_DST_TOO_SMALL;
@@ -520,6 +531,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
                                     uint32_t *done_flags_host, int32_t flags_cap, int32_t *n_chunks_out,
                                     aaf_kv_xfer_desc *out_desc, void *stream) {
     if (!p || !dst_host || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
     if (!aligned16(staging_dev) || t0 < 0 || t0 >= t1 || t1 > p->len[ctx]) return AAF_ERR_INVALID_ARG;
     const long long n = t1 - t0;
@@ -532,7 +544,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     const int n_chunks = (n_slots + per_chunk - 1) / per_chunk;
     if (done_flags_host && flags_cap < n_chunks) return AAF_ERR_DST_TOO_SMALL;
     DeviceGuard guard(p->device);
-    if (!ensure_xfer_stream(p)) return AAF_ERR_CUDA;
+    if (!ensure_xfer_stream(p)) return broke(p);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
     if (done_flags_host)
@@ -541,7 +553,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     if (launch_plan_materialize(p->g, ps.view, ctx, t0, t1, static_cast<char *>(staging_dev), p->clock + 1,
                                 p->meta_stream) != cudaSuccess ||
         !end_plan(p, ps, st))
-        return AAF_ERR_CUDA;
+        return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     bool ok = true;
@@ -563,7 +575,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
     // the caller's stream is complete only when the last chunk has landed
     cudaEvent_t fin = order_event(p);
     ok = ok && fin && cudaEventRecord(fin, p->xfer_stream) == cudaSuccess && cudaStreamWaitEvent(st, fin, 0) == cudaSuccess;
-    if (!ok) return AAF_ERR_CUDA;
+    if (!ok) return broke(p);
     if (n_chunks_out) *n_chunks_out = n_chunks;
     if (out_desc) fill_desc(p, out_desc, t0, n);
     return AAF_OK;
@@ -574,6 +586,7 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     if (!p || !src_host || !desc || !out_ctx || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0 ||
         !aligned16(staging_dev))
         return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (!compatible(p, desc)) return AAF_ERR_INCOMPAT;
     const long long n = desc->n_tokens;
     if (n < 1) return AAF_ERR_INVALID_ARG;
@@ -583,7 +596,7 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     const int c = smallest_free_ctx(p);
     if (c < 0) return AAF_ERR_OOM_CTX;
     DeviceGuard guard(p->device);
-    if (!ensure_xfer_stream(p)) return AAF_ERR_CUDA;
+    if (!ensure_xfer_stream(p)) return broke(p);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int rc0 = ensure_free(p, nb, st);
     if (rc0 != AAF_OK) return rc0;
@@ -597,7 +610,7 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     ok = ok && launch_plan_import(p->g, ps.view, c, n, static_cast<const char *>(staging_dev), p->clock + 1,
                                   p->meta_stream) == cudaSuccess &&
          end_plan(p, ps, st);
-    if (!ok) return AAF_ERR_CUDA;
+    if (!ok) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= nb;
@@ -617,11 +630,12 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
         ok = ok && run_copy(p, ps, AAF_OP_IMPORT, (int)(s1 - s0), hi - lo, st, (int)s0) == AAF_OK;
     }
     end_copy(p, ps, st);
-    return ok ? AAF_OK : AAF_ERR_CUDA;
+    return ok ? AAF_OK : broke(p);
 }
 
 int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream) {
     if (!p || !out_children || k < 1) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (!is_live(p, parent)) return AAF_ERR_BAD_CTX;
     if (k > p->lay.max_batch) return AAF_ERR_TOO_MANY;
     if (p->g.max_ctx - p->live_ctx < k) return AAF_ERR_OOM_CTX;
@@ -637,7 +651,7 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
     const long long T = p->len[parent];
     const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, children, p->clock + 1, p->meta_stream);
     release_args(p, p->meta_stream);
-    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    if (e != cudaSuccess) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     for (int j = 0; j < k; ++j) {
@@ -651,6 +665,7 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
 int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
                   const void *const *src_dev, void *stream) {
     if (!p || n < 1 || !ctxs || !n_new || !src_dev) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
     for (int i = 0; i < n; ++i) {
         if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
@@ -713,7 +728,7 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
     const cudaError_t e = launch_plan_append(p->g, ps.view, ent, n, (int)slots, p->lay.max_batch, 0, p->clock + 1,
                                              p->meta_stream);
     release_args(p, p->meta_stream);
-    if (e != cudaSuccess || !end_plan(p, ps, st)) return AAF_ERR_CUDA;
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= charge;
@@ -726,6 +741,7 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
 int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
                    void *stream) {
     if (!p || m < 1 || !segs || !out_ctx || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (m > p->lay.max_batch) return AAF_ERR_TOO_MANY;
     for (int i = 0; i < m; ++i)
         if (!is_live(p, segs[i])) return AAF_ERR_BAD_CTX;
@@ -773,7 +789,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, m, (int)work, (int)fresh, (int)slots, c,
                                               p->clock + 1, p->meta_stream);
     release_args(p, p->meta_stream);
-    if (e != cudaSuccess || !end_plan(p, ps, st)) return AAF_ERR_CUDA;
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
     p->free_lb -= fresh;
@@ -787,6 +803,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
 
 int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {
     if (!p || n < 1 || !ctxs) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
     for (int i = 0; i < n; ++i)
         if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
@@ -813,7 +830,7 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
     int n_launches = 0;
     const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, p->clock + 1, &n_launches, p->meta_stream);
     release_args(p, p->meta_stream);
-    if (e != cudaSuccess) return AAF_ERR_CUDA;
+    if (e != cudaSuccess) return broke(p);
     p->clock += 1;
     p->meta_launches += n_launches;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] = -1;
@@ -824,6 +841,7 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
 int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gamma, int64_t budget_blocks,
                            aaf_ctx_t *out_victims, int32_t cap, int32_t *n_victims, void *stream) {
     if (!p || !out_victims || !n_victims || budget_blocks < 0) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     if (!(alpha == alpha && beta == beta && gamma == gamma) || alpha - alpha != 0.0 || beta - beta != 0.0 ||
         gamma - gamma != 0.0)
         return AAF_ERR_INVALID_ARG;  // NaN or infinite weights
@@ -833,10 +851,10 @@ int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gam
     p->last_stream = st;
     if (launch_evict_to_budget(p->g, p->s, alpha, beta, gamma, budget_blocks, p->clock + 1, p->result,
                                p->meta_stream) != cudaSuccess)
-        return AAF_ERR_CUDA;
+        return broke(p);
     p->meta_launches += 1;
     // the victims are chosen on the device; the host mirror needs them before the next call
-    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess) return AAF_ERR_CUDA;
+    if (cudaStreamSynchronize(p->meta_stream) != cudaSuccess) return broke(p);
     p->clock += 1;
     const int nv = p->result[0];
     for (int i = 0; i < nv; ++i) {
@@ -862,6 +880,7 @@ int aaf_kv_catalog_rows(aaf_kv_pool *p, int32_t *n_states, int64_t *n_block_rows
 
 int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void *stream) {
     if (!p || !cols) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
     int32_t ns = 0;
     int64_t rows = 0;
     aaf_kv_catalog_rows(p, &ns, &rows);
@@ -878,7 +897,7 @@ int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void 
     cudaEvent_t done = order_event(p);
     if (launch_export_catalog(p->g, p->s, *cols, ns, rows, p->meta_stream) != cudaSuccess || !done ||
         cudaEventRecord(done, p->meta_stream) != cudaSuccess || cudaStreamWaitEvent(st, done, 0) != cudaSuccess)
-        return AAF_ERR_CUDA;
+        return broke(p);
     p->meta_launches += rows > 0 ? 2 : 1;
     return AAF_OK;
 }

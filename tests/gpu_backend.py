@@ -1,6 +1,6 @@
 """The CUDA library behind the replay-backend interface of ``workloads.replay`` / ``workloads.churn``.
 
-Harness code for tests and benchmarks: it owns a ``KVPool``, produces payloads on the device with
+Harness code for the tests, the smoke check and the benchmark (not part of the product package): it owns a ``KVPool``, produces payloads on the device with
 ``workloads.fill`` and forwards every operator to the library.  Nothing is computed here.
 """
 from __future__ import annotations
@@ -12,7 +12,8 @@ from workloads.configs import Geometry
 
 
 def snapshot(o) -> dict:
-    """Everything observable about a pool except its bytes."""
+    """Everything observable about a pool except its bytes (works on the library's KVPool and on the oracle's
+    PagedOracle: both expose the same introspection names)."""
     live = o.live_ctxs()
     return {
         "lens": {c: o.ctx_len(c) for c in live},
@@ -29,7 +30,7 @@ class GpuBackend:
                  staging_tokens: int = 0):
         import torch
 
-        from .binding import KVPool
+        from paper_2607_10987_b200.binding import KVPool
 
         self.g, self.torch, self.seed_ = g, torch, seed
         self._big = None

@@ -79,17 +79,6 @@ class OracleBackend:
         return snapshot(self.o)
 
 
-def snapshot(o) -> dict:
-    """Everything observable about a pool except its bytes."""
-    live = o.live_ctxs()
-    return {
-        "lens": {c: o.ctx_len(c) for c in live},
-        "tables": {c: o.table(c).tolist() for c in live},
-        "refcounts": o.refcounts().tolist(),
-        "free_list": o.free_list().tolist(),
-    }
-
-
 def check_conservation(snap: dict, n_blocks: int, block_size: int):
     """Reference-count conservation, recounted from the tables alone:
     refcount[b] = number of table entries naming b; free ring = exactly the
@@ -184,4 +173,4 @@ def expected_bytes(seed: int, g: Geometry, tokens, layers=None) -> np.ndarray:
     return out.view(np.uint8).reshape(len(layers), 2, len(tokens), g.row)
 
 
-from paper_2607_10987_b200.replay_backend import GpuBackend  # noqa: E402,F401  (re-exported for the tests)
+from tests.gpu_backend import GpuBackend, snapshot  # noqa: E402,F401  (re-exported for the tests)

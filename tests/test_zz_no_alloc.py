@@ -3,8 +3,9 @@
 aaf_kv_materialize_noalloc serves callers that may not call cudaMalloc (all device memory already
 committed to their own pool, a path that cannot afford an allocation's synchronisation, code that
 is only handed pointers).  Its scratch is a fixed array inside the library that every call on the
-device shares and that keeps the previous call's contents, so the check runs two different
-requests back to back and compares each, byte for byte, with aaf_kv_materialize.
+device shares and that keeps the previous call's contents, so the check runs different
+requests back to back and compares each, byte for byte, with aaf_kv_materialize and with the CPU
+oracle's materialize of the same context.
 """
 from __future__ import annotations
 
@@ -23,11 +24,14 @@ def test_noalloc_gather_matches_materialize_twice_in_a_row():
     from paper_2607_10987_b200 import KVPool, binding
     from workloads import configs, fill
 
+    from tests.helpers import OracleBackend
+
     entry.build()
     g = configs.Geometry(3, 8, 128, 16, 2, 512, 8, 128)
     seed = 424242
     pool = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, g.n_blocks, g.max_ctx,
                   g.max_blocks_per_ctx, free_order=configs.free_order(seed, g.n_blocks))
+    cpu = OracleBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks))
     dev = pool.device
     fill.fill_torch(seed, 0, 0, g.pool_bytes // 2, dev, out=pool.pool.view(torch.int16))
     ctxs = []
@@ -35,6 +39,7 @@ def test_noalloc_gather_matches_materialize_twice_in_a_row():
         buf = fill.fill_torch(seed, stream_id, 0, g.n_layers * 2 * n * g.row // 2, dev).view(torch.uint8)
         st, c = pool.imp(buf, n)
         assert st == 0
+        assert cpu.imp(cpu.payload(seed, stream_id, n), n) == (0, c)
         ctxs.append((c, n))
     stream = C.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
 
@@ -56,6 +61,22 @@ def test_noalloc_gather_matches_materialize_twice_in_a_row():
         assert st == binding.AAF_OK
         torch.cuda.synchronize()
         assert torch.equal(got, want[: got.numel()]), (c, t0, t1)
+        st, oracle_bytes = cpu.materialize(c, t0, t1)
+        assert st == 0 and np.array_equal(got.cpu().numpy(), oracle_bytes), (c, t0, t1)
+
+    # a pinned table is uploaded asynchronously: it may be overwritten only after the stream has run the call
+    c, n = ctxs[1]
+    table = pool.table(c)
+    pinned = torch.from_numpy(table.copy()).pin_memory()
+    out = torch.full((n * g.bpt,), 0x5A, dtype=torch.uint8, device=dev)
+    st = binding.aaf_kv_materialize_noalloc(pool.pool.data_ptr(), g.layer_stride, g.n_layers, g.n_kv_heads,
+                                            g.head_dim, g.block_size, g.elt_bytes, g.n_blocks,
+                                            C.cast(pinned.data_ptr(), C.POINTER(C.c_int32)), len(table), 0, n,
+                                            out.data_ptr(), out.numel(), stream)
+    assert st == binding.AAF_OK
+    torch.cuda.synchronize()
+    pinned.fill_(-1)
+    assert np.array_equal(out.cpu().numpy(), cpu.materialize(c, 0, n)[1])
 
     # beyond the built-in scratch: rejected with its own status, nothing launched
     big_blocks = binding.AAF_NOALLOC_MAX_BLOCKS + 1
