@@ -227,6 +227,20 @@ int aaf_kv_materialize_host(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin,
 int aaf_kv_import_host(aaf_kv_pool *pool, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
                        size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream);
 
+/* append with the continuation tokens in HOST memory -- Alg. "KV-Resume" (register continuation KV)
+ * fed from the transport's host end (Sec. 5.4).  Same result as aaf_kv_append, but src_host[i] (host,
+ * transfer layout [L][2][n_new[i]][H][D]; pinned memory for a truly asynchronous copy) is first
+ * uploaded into staging_dev (device, caller-owned scratch, >= sum(n_new) * bpt bytes, 16-byte
+ * aligned), entry after entry, on a library-owned copy stream; the scatter on `stream` waits for the
+ * upload.  The upload does NOT wait for work already queued on `stream`, except for the scatter of
+ * the previous aaf_kv_append_host of this pool: staging_dev must be scratch that nothing else has in
+ * use, so that the upload can overlap whatever `stream` is still doing (e.g. a transfer buffer on its
+ * way back to the host).  Host buffers and staging_dev must stay untouched until `stream` has run
+ * the call.  Errors as aaf_kv_append, plus DST_TOO_SMALL for a staging buffer that is too small;
+ * after an error the contents of staging_dev are undefined. */
+int aaf_kv_append_host(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
+                       const void *const *src_host, void *staging_dev, size_t staging_bytes, void *stream);
+
 /* Chunked, overlapped forms of the host transfer (Sec. 5.4: the transport overlaps communication
  * with computation, and consumers may start as blocks arrive).  The token range is cut into chunks
  * of chunk_tokens tokens (a multiple of block_size, counted from the block that holds tok_begin);
@@ -239,7 +253,10 @@ int aaf_kv_import_host(aaf_kv_pool *pool, const void *src_host, const aaf_kv_xfe
  *   blocks [c * chunk_tokens / BS, ...) of the range in every (layer, K/V) plane of dst_host.
  *   *n_chunks_out (host, may be NULL) receives the number of chunks.  `stream` is complete only
  *   when the last chunk has landed.
- *   import: blocks are allocated up front; chunk c is scattered as soon as it has arrived.
+ *   import: blocks are allocated up front; chunk c is scattered as soon as it has arrived.  The upload
+ *   runs on the library's upload stream (uploads of this pool arrive in call order) and does NOT wait for
+ *   work already queued on `stream`, except for the scatter of the previous aaf_kv_import_host_chunked:
+ *   staging_dev must be scratch that nothing else has in use.
  * Errors as for the unchunked forms, plus INVALID_ARG for a chunk_tokens that is not a positive
  * multiple of block_size and DST_TOO_SMALL for too few flags. */
 int aaf_kv_materialize_host_chunked(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end,

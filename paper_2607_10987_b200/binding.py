@@ -78,6 +78,7 @@ SYMBOLS = {
     "aaf_kv_evict": (C.c_int, [_vp, _i32, _p32, _vp]),
     "aaf_kv_materialize_host": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _p32, _vp]),
+    "aaf_kv_append_host": (C.c_int, [_vp, _i32, _p32, _p32, C.POINTER(_vp), _vp, _sz, _vp]),
     "aaf_kv_materialize_host_chunked": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, _i32, C.POINTER(C.c_uint32),
                                                   _i32, _p32, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host_chunked": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _i32, _p32, _vp]),
@@ -138,6 +139,8 @@ def aaf_kv_materialize_host(pool, ctx, t0, t1, dst_host, dst_bytes, staging, sta
     return _fn("aaf_kv_materialize_host")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream)
 def aaf_kv_import_host(pool, src_host, desc, staging, staging_bytes, out_ctx, stream):
     return _fn("aaf_kv_import_host")(pool, src_host, desc, staging, staging_bytes, out_ctx, stream)
+def aaf_kv_append_host(pool, n, ctxs, n_new, srcs_host, staging, staging_bytes, stream):
+    return _fn("aaf_kv_append_host")(pool, n, ctxs, n_new, srcs_host, staging, staging_bytes, stream)
 def aaf_kv_materialize_host_chunked(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, chunk_tokens,
                                     done_flags, flags_cap, n_chunks_out, out_desc, stream):
     return _fn("aaf_kv_materialize_host_chunked")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes,
@@ -270,6 +273,15 @@ class KVPool:
         b = (C.c_int32 * max(n, 1))(*n_new)
         ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in bufs])
         return aaf_kv_append(self.h, n, a, b, ptrs, self._stream()), None
+
+    def append_host(self, ctxs, n_new, host_bufs, staging):
+        """host_bufs: one (pinned) host tensor per entry; staging: device scratch for all of them."""
+        n = len(ctxs)
+        a = (C.c_int32 * max(n, 1))(*ctxs)
+        b = (C.c_int32 * max(n, 1))(*n_new)
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in host_bufs])
+        return aaf_kv_append_host(self.h, n, a, b, ptrs, staging.data_ptr(), staging.numel() * staging.element_size(),
+                                  self._stream())
 
     def compose(self, segs, flags=0):
         m = len(segs)

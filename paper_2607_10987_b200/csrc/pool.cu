@@ -125,7 +125,13 @@ struct aaf_kv_pool {
     std::vector<TimedLaunch> pending;
     std::vector<cudaEvent_t> spare_events;
     // chunked host transfers: a second stream for the PCIe copies and ordering events
-    cudaStream_t xfer_stream = nullptr;
+    // chunked / host-buffer transfers: one library-owned stream per PCIe direction, so that uploads queue behind
+    // each other in call order (the first one needed arrives first) while a download runs beside them
+    cudaStream_t xfer_stream = nullptr;     // device -> host (aaf_kv_materialize_host_chunked)
+    cudaStream_t upload_stream = nullptr;   // host -> device (aaf_kv_import_host_chunked, aaf_kv_append_host)
+    // the scatter launches of the last upload call per staging role have read their staging buffer
+    cudaEvent_t upload_reader_done = nullptr, import_reader_done = nullptr;
+    bool upload_reader_pending = false, import_reader_pending = false;
     std::vector<cudaEvent_t> order_events;  // created on demand, reused round-robin
     size_t next_order_event = 0;
 };
@@ -343,6 +349,17 @@ bool ensure_xfer_stream(aaf_kv_pool *p) {
     if (p->xfer_stream) return true;
     return cudaStreamCreateWithFlags(&p->xfer_stream, cudaStreamNonBlocking) == cudaSuccess;
 }
+bool ensure_upload_stream(aaf_kv_pool *p) {
+    if (!p->upload_stream && cudaStreamCreateWithFlags(&p->upload_stream, cudaStreamNonBlocking) != cudaSuccess)
+        return false;
+    if (!p->upload_reader_done &&
+        cudaEventCreateWithFlags(&p->upload_reader_done, cudaEventDisableTiming) != cudaSuccess)
+        return false;
+    if (!p->import_reader_done &&
+        cudaEventCreateWithFlags(&p->import_reader_done, cudaEventDisableTiming) != cudaSuccess)
+        return false;
+    return true;
+}
 
 // column slab [col0, col0 + cnt) tokens of an n-token transfer buffer: 2L rows of cnt*row bytes, pitch n*row
 cudaError_t copy_slab(aaf_kv_pool *p, char *dst, const char *src, long long n, long long col0, long long cnt,
@@ -468,6 +485,12 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
         cudaStreamSynchronize(p->xfer_stream);
         cudaStreamDestroy(p->xfer_stream);
     }
+    if (p->upload_stream) {
+        cudaStreamSynchronize(p->upload_stream);
+        cudaStreamDestroy(p->upload_stream);
+    }
+    if (p->upload_reader_done) cudaEventDestroy(p->upload_reader_done);
+    if (p->import_reader_done) cudaEventDestroy(p->import_reader_done);
     for (auto e : p->order_events) cudaEventDestroy(e);
     for (int i = 0; i < 2; ++i) {
         if (p->plan_done[i]) cudaEventDestroy(p->plan_done[i]);
@@ -596,16 +619,15 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
     const int c = smallest_free_ctx(p);
     if (c < 0) return AAF_ERR_OOM_CTX;
     DeviceGuard guard(p->device);
-    if (!ensure_xfer_stream(p)) return broke(p);
+    if (!ensure_upload_stream(p)) return broke(p);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int rc0 = ensure_free(p, nb, st);
     if (rc0 != AAF_OK) return rc0;
     p->last_stream = st;
-    // the PCIe stream may only overwrite the staging buffer after everything already queued on the
-    // caller's stream (earlier readers of that buffer) has run
-    cudaEvent_t start = order_event(p);
-    bool ok = start && cudaEventRecord(start, st) == cudaSuccess &&
-              cudaStreamWaitEvent(p->xfer_stream, start, 0) == cudaSuccess;
+    // staging_dev is this call's scratch: the only earlier reader the library knows of is the scatter of the
+    // previous aaf_kv_import_host_chunked, so the upload waits for that and for nothing else on `stream`
+    bool ok = !p->import_reader_pending ||
+              cudaStreamWaitEvent(p->upload_stream, p->import_reader_done, 0) == cudaSuccess;
     const PlanSlot ps = begin_plan(p);
     ok = ok && launch_plan_import(p->g, ps.view, c, n, static_cast<const char *>(staging_dev), p->clock + 1,
                                   p->meta_stream) == cudaSuccess &&
@@ -622,15 +644,18 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
         const long long s1 = std::min<long long>(nb, s0 + per_chunk);
         const long long lo = s0 * BS, hi = std::min<long long>(n, s1 * BS);
         ok = copy_slab(p, static_cast<char *>(staging_dev), static_cast<const char *>(src_host), n, lo, hi - lo,
-                       cudaMemcpyHostToDevice, p->xfer_stream) == cudaSuccess;
+                       cudaMemcpyHostToDevice, p->upload_stream) == cudaSuccess;
         cudaEvent_t ev = order_event(p);
-        ok = ok && ev && cudaEventRecord(ev, p->xfer_stream) == cudaSuccess &&
+        ok = ok && ev && cudaEventRecord(ev, p->upload_stream) == cudaSuccess &&
              cudaStreamWaitEvent(st, ev, 0) == cudaSuccess;
         // scatter of the chunk that has arrived, while the next one crosses PCIe
         ok = ok && run_copy(p, ps, AAF_OP_IMPORT, (int)(s1 - s0), hi - lo, st, (int)s0) == AAF_OK;
     }
     end_copy(p, ps, st);
-    return ok ? AAF_OK : broke(p);
+    ok = ok && cudaEventRecord(p->import_reader_done, st) == cudaSuccess;
+    if (!ok) return broke(p);
+    p->import_reader_pending = true;
+    return AAF_OK;
 }
 
 int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream) {
@@ -662,25 +687,35 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
     return AAF_OK;
 }
 
+// everything about an append batch that the host can check without the device
+static int append_check(const aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new) {
+    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    for (int i = 0; i < n; ++i) {
+        if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
+        if (n_new[i] < 1) return AAF_ERR_INVALID_ARG;
+    }
+    std::vector<int> sorted(ctxs, ctxs + n);
+    std::sort(sorted.begin(), sorted.end());
+    if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AAF_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i)
+        if (nblk_of(p, p->len[ctxs[i]] + n_new[i]) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+    return AAF_OK;
+}
+
 int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
                   const void *const *src_dev, void *stream) {
     if (!p || n < 1 || !ctxs || !n_new || !src_dev) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
-    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
-    for (int i = 0; i < n; ++i) {
-        if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
-        if (n_new[i] < 1 || !aligned16(src_dev[i])) return AAF_ERR_INVALID_ARG;
-    }
     {
-        std::vector<int> sorted(ctxs, ctxs + n);
-        std::sort(sorted.begin(), sorted.end());
-        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AAF_ERR_INVALID_ARG;
+        const int rc = append_check(p, n, ctxs, n_new);
+        if (rc != AAF_OK) return rc;
     }
+    for (int i = 0; i < n; ++i)
+        if (!aligned16(src_dev[i])) return AAF_ERR_INVALID_ARG;
     const int BS = p->g.BS;
     long long worst = 0, slots = 0, append_tokens = 0;  // append_tokens: new tokens plus the copy-on-write worst case
     for (int i = 0; i < n; ++i) {
         const long long T = p->len[ctxs[i]];
-        if (nblk_of(p, T + n_new[i]) > p->g.max_blk) return AAF_ERR_TOO_LONG;
         append_tokens += n_new[i] + T % BS;
         worst += (T % BS ? 1 : 0) + nblk_of(p, T + n_new[i]) - nblk_of(p, T);
         slots += 1 + nblk_of(p, T + n_new[i]) - T / BS;
@@ -736,6 +771,46 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
     const int rc_copy = run_copy(p, ps, AAF_OP_APPEND, (int)slots, append_tokens, st);
     end_copy(p, ps, st);
     return rc_copy;
+}
+
+int aaf_kv_append_host(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
+                       const void *const *src_host, void *staging_dev, size_t staging_bytes, void *stream) {
+    if (!p || n < 1 || !ctxs || !n_new || !src_host || !aligned16(staging_dev)) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
+    {
+        const int rc = append_check(p, n, ctxs, n_new);
+        if (rc != AAF_OK) return rc;
+    }
+    unsigned long long need_bytes = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!src_host[i]) return AAF_ERR_INVALID_ARG;
+        need_bytes += (unsigned long long)n_new[i] * (unsigned long long)bpt_of(p);
+    }
+    if ((unsigned long long)staging_bytes < need_bytes) return AAF_ERR_DST_TOO_SMALL;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!ensure_upload_stream(p)) return AAF_ERR_CUDA;
+    // the staging buffer is this call's scratch: the only earlier reader the library knows of is the copy launch
+    // of the previous aaf_kv_append_host, so the upload waits for that one and for nothing else on `stream`
+    bool ok = !p->upload_reader_pending || cudaStreamWaitEvent(p->upload_stream, p->upload_reader_done, 0) == cudaSuccess;
+    std::vector<const void *> dev_ptrs((size_t)n);
+    char *cursor = static_cast<char *>(staging_dev);
+    for (int i = 0; i < n && ok; ++i) {  // one copy per entry, back to back on the upload stream
+        const size_t bytes = (size_t)n_new[i] * (size_t)bpt_of(p);
+        ok = cudaMemcpyAsync(cursor, src_host[i], bytes, cudaMemcpyHostToDevice, p->upload_stream) == cudaSuccess;
+        dev_ptrs[(size_t)i] = cursor;
+        cursor += bytes;
+    }
+    cudaEvent_t arrived = order_event(p);
+    ok = ok && arrived && cudaEventRecord(arrived, p->upload_stream) == cudaSuccess &&
+         cudaStreamWaitEvent(st, arrived, 0) == cudaSuccess;
+    if (!ok) return broke(p);
+    const int rc = aaf_kv_append(p, n, ctxs, n_new, dev_ptrs.data(), stream);
+    if (rc == AAF_OK) {
+        if (cudaEventRecord(p->upload_reader_done, st) != cudaSuccess) return broke(p);
+        p->upload_reader_pending = true;
+    }
+    return rc;
 }
 
 int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,

@@ -46,6 +46,35 @@ def test_host_buffer_forms_match_the_oracle():
     assert gpu.snapshot() == cpu.snapshot()
 
 
+def test_append_from_host_buffers_matches_the_oracle():
+    """aaf_kv_append_host: continuation tokens uploaded from pinned host memory, copy-on-write included; two
+    calls in a row reuse the same staging buffer (the second upload must wait for the first scatter)."""
+    order = configs.free_order(SEED, G.n_blocks)
+    gpu = GpuBackend(G, SEED, free_order=order)
+    cpu = OracleBackend(G, SEED, free_order=order)
+    n = 203  # 203 = 12 * 16 + 11: the tail block holds 11 rows and is shared after the fork
+    for be in (gpu, cpu):
+        st, root = be.imp(be.payload(SEED, 1, n), n)
+        assert (st, root) == (0, 0)
+        st, kids = be.fork(root, 3)
+        assert st == 0 and kids == [1, 2, 3]
+    staging = torch.empty(64 * G.bpt, dtype=torch.uint8, device=gpu.o.device)
+    for rnd, n_new in enumerate(([7, 21, 1], [16, 5, 30])):
+        payloads = [cpu.payload(SEED, 10 * rnd + 2 + i, k) for i, k in enumerate(n_new)]
+        hosts = [torch.from_numpy(p.copy()).pin_memory() for p in payloads]
+        assert gpu.o.append_host(kids, n_new, hosts, staging) == 0
+        assert cpu.append(kids, n_new, payloads)[0] == 0
+        assert gpu.snapshot() == cpu.snapshot()
+    torch.cuda.synchronize()
+    assert np.array_equal(gpu.pool_layers(range(G.n_layers)), cpu.o.pool_view())
+    assert gpu.o.stats()["cow_count"] == cpu.o.stats()["cow_count"] == 3
+    # argument checks: staging too small, a dead handle, a null host pointer
+    hosts = [torch.zeros(G.bpt, dtype=torch.uint8).pin_memory() for _ in range(3)]
+    assert gpu.o.append_host(kids, [1, 1, 1], hosts, staging[: 2 * G.bpt]) == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.append_host([7], [1], hosts[:1], staging) == binding.AAF_ERR_BAD_CTX
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+
+
 def test_incompatible_descriptor_is_refused_and_changes_nothing():
     gpu = GpuBackend(G, SEED)
     buf = gpu.payload(SEED, 1, 40)

@@ -25,11 +25,12 @@ WORKER = textwrap.dedent(
     t = torch.tensor([float(moved)])
     dist.all_reduce(t)
     assert t.item() == world * moved
-    ms = torch.tensor([10.0 + rank])         # rank-dependent step time: the job reports the slowest
-    dist.barrier()
-    dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    assert ms.item() == 10.0 + world - 1
-    value = world * moved / (ms.item() * 1e-3) / 1e9
+    # the benchmark's own control plane: barrier, then the slowest rank's time is the job's time
+    cl = bench.Cluster(torch, dist, "cpu", world, "gloo")
+    cl.barrier()
+    ms = cl.max_ms(10.0 + rank)              # rank-dependent step time: the job reports the slowest
+    assert ms == 10.0 + world - 1
+    value = world * moved / (ms * 1e-3) / 1e9
     if rank == 0:
         print(json.dumps({"value": value, "n_gpus": world, "scaling": "weak"}))
     dist.destroy_process_group()
