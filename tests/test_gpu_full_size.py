@@ -11,9 +11,12 @@ import numpy as np
 import pytest
 import torch
 
+from tests.helpers import GpuBackend, check_conservation
 from tests.test_gpu_parity import lockstep
+from tests.value_check import ShadowBackend
 from workloads import configs
 from workloads.configs import Geometry
+from workloads.replay import replay
 
 pytestmark = pytest.mark.gpu
 
@@ -88,3 +91,78 @@ def test_cow_stress_1024_children_8b_rows():
     assert gpu.evict([0])[0] == 0 and cpu.evict([0])[0] == 0
     assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
     assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Convention-free checks at full size, ALL layers: the value model (contexts are token sequences; no blocks, no
+# reference counts, no free list) runs beside the library; every materialised buffer and, at the end, every live
+# context is compared in every (layer, K/V) plane with bytes regenerated on the device from the fill function.
+# These tests do not use the paged oracle: they hold whatever block ids the library hands out.  Reference-count
+# conservation (refcount = number of table entries naming the block, free ring = exactly the unreferenced blocks)
+# is recounted from the library's own tables.
+
+
+def value_model_run(g, seed, ops, max_batch=0, staging_tokens=0):
+    gpu = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), init_fill=False, max_batch=max_batch,
+                     staging_tokens=staging_tokens)
+    sh = ShadowBackend(gpu)
+    n_bufs = 0
+    for i, op, st, res, _ in replay(ops, sh, seed):
+        assert st == 0, (i, op, st)
+        if op["op"] == "materialize":
+            sh.check_buffer(seed, res)
+            n_bufs += 1
+    sh.check_all_live(seed)
+    check_conservation(gpu.snapshot(), g.n_blocks, g.block_size)
+    assert gpu.o.sync_status() == 0
+    return sh, n_bufs
+
+
+def test_config2_llama8b_value_model_all_layers():
+    g, seed, ops = configs.config2(True)
+    if not _fits(g, 12):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    sh, n_bufs = value_model_run(g, seed, ops)
+    assert n_bufs == 18 and len(sh.vm.ctx) == 18
+    assert sh.planes_checked == 64 * (n_bufs + 18)
+
+
+@pytest.mark.parametrize("copy_all", [False, True])
+def test_config3_compose_levels_value_model_all_layers(copy_all):
+    g, seed, ops, lens = configs.config3(configs.LLAMA8B, copy_all=copy_all)
+    if not _fits(g, 16):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    sh, n_bufs = value_model_run(g, seed, ops)
+    assert n_bufs == 2 and len(sh.vm.ctx) == 16 + 8 + 4 + 2
+    # the tree and the flat composition are the same sequence
+    assert sh.vm.ctx[max(sh.vm.ctx)] == sh.vm.ctx[max(sh.vm.ctx) - 1] and len(sh.vm.ctx[max(sh.vm.ctx)]) == sum(lens)
+
+
+def test_config4_llama70b_value_model_all_layers():
+    g, seed, ops = configs.config4(True)
+    if not _fits(g, 40):
+        pytest.skip("not enough free device memory for the 40 GiB pool plus 10 GiB buffers")
+    sh, n_bufs = value_model_run(g, seed, ops)
+    assert n_bufs == 10 and len(sh.vm.ctx) == 10
+    assert sh.planes_checked == 160 * (n_bufs + 10)
+
+
+def test_cow_stress_value_model_all_layers():
+    g = Geometry(32, 8, 128, 16, 2, 4096, 1100, 1024)
+    ops = configs.cow_stress_ops(context_tokens=8187, n_children=64)  # 64 children: every one compared in full
+    sh, _ = value_model_run(g, configs.SEED_BASE + 6, ops, max_batch=1024)
+    assert len(sh.vm.ctx) == 65 and sh.gpu.o.stats()["cow_count"] == 64
+
+
+def test_value_check_detects_one_wrong_byte():
+    """The all-layer comparison is not vacuous: one flipped byte in the last layer of a buffer fails it."""
+    g = Geometry(4, 8, 128, 16, 2, 64, 4, 32)
+    seed = 5
+    gpu = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), init_fill=False)
+    sh = ShadowBackend(gpu)
+    st, c = sh.imp(sh.payload(seed, 1, 100), 100)
+    st, buf = sh.materialize(c, 3, 97)
+    sh.check_buffer(seed, buf)
+    buf.dev[buf.dev.numel() - 7] ^= 1
+    with pytest.raises(AssertionError, match="layer 3 kv 1"):
+        sh.check_buffer(seed, buf)

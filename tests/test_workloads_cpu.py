@@ -60,3 +60,34 @@ def test_config3_lengths_and_levels():
     g, seed, ops, lens = configs.config3(configs.LLAMA8B)
     assert len(lens) == 16 and all(1024 <= n <= 4096 and n % 16 for n in lens)
     assert sum(1 for o in ops if o["op"] == "compose") == 8 + 4 + 1 + 1
+
+
+def test_device_side_expected_bytes_equal_the_numpy_ones():
+    """The torch routine that regenerates a token sequence's transfer-buffer bytes (used on the GPU to compare
+    every layer at full size) against the numpy one, on CPU tensors, with tokens from several payloads and a
+    windowed payload."""
+    import torch
+
+    from tests.helpers import expected_bytes
+    from tests.value_check import expected_plane, token_tensor
+    from workloads import fill
+    from workloads.configs import Geometry
+
+    g = Geometry(3, 2, 8, 4, 2, 16, 4, 8)
+    seed = 77
+    tokens = [(1, t, 9, 0) for t in range(2, 9)] + [(5, t, 4, 0) for t in range(4)] + [(1, 0, 9, 0)]
+    want = expected_bytes(seed, g, [tk[:3] for tk in tokens])
+    q = fill.quantile_table_torch("cpu")
+    tt = token_tensor(seed, tokens, "cpu")
+    hd = g.row // 2
+    for l in range(g.n_layers):
+        for kv in range(2):
+            got = expected_plane(tt, l, kv, hd, q).numpy().view(np.uint16)
+            assert np.array_equal(got.view(np.uint8).reshape(len(tokens), g.row), want[l, kv])
+    # a windowed payload: element index shifted by the window's base
+    base, n = 40, 6
+    tt = token_tensor(seed, [(1, t, n, base) for t in range(n)], "cpu")
+    flat = fill.fill_np(seed, 1, base, g.n_layers * 2 * n * hd).reshape(g.n_layers, 2, n, hd)
+    for l in range(g.n_layers):
+        for kv in range(2):
+            assert np.array_equal(expected_plane(tt, l, kv, hd, q).numpy().view(np.uint16), flat[l, kv])

@@ -75,6 +75,35 @@ def _s64(v: int) -> int:
     return v - (1 << 64) if v >= (1 << 63) else v
 
 
+def _lsr(x, s):
+    """logical right shift of an int64 tensor (arithmetic shift, then mask)"""
+    return (x >> s) & ((1 << (64 - s)) - 1)
+
+
+def quantile_table_torch(device):
+    import torch
+
+    return torch.from_numpy(quantile_table().view(np.int16).copy()).to(device)
+
+
+def fill_torch_at(key, idx, q):
+    """int16 tensor shaped like ``idx``: elements ``idx`` (int64 tensor) of the stream(s) whose key(s) ``key`` is
+    an int (one stream) or an int64 tensor broadcastable against ``idx`` (``key_s64`` of each element's stream).
+    Wrapping int64 arithmetic; ``q`` = quantile_table_torch(device)."""
+    x = idx * _s64(_ODD) + key
+    x = x ^ _lsr(x, 30)
+    x = x * _s64(_M1)
+    x = x ^ _lsr(x, 27)
+    x = x * _s64(_M2)
+    x = x ^ _lsr(x, 31)
+    return q[_lsr(x, 48)]
+
+
+def key_s64(seed: int, stream: int) -> int:
+    """the stream key as a two's-complement int64 (what fill_torch_at adds)"""
+    return _s64(stream_key(seed, stream))
+
+
 def fill_torch(seed: int, stream: int, start: int, count: int, device, out=None, chunk: int = 1 << 26):
     """int16 tensor [count] on ``device`` holding the same bit patterns as fill_np.
 
@@ -86,22 +115,12 @@ def fill_torch(seed: int, stream: int, start: int, count: int, device, out=None,
     if out is None:
         out = torch.empty(count, dtype=torch.int16, device=device)
     assert out.numel() == count and out.dtype == torch.int16
-    q = torch.from_numpy(quantile_table().view(np.int16).copy()).to(device)
-    key = _s64(stream_key(seed, stream))
-
-    def lsr(x, s):
-        return (x >> s) & ((1 << (64 - s)) - 1)
-
+    q = quantile_table_torch(device)
+    key = key_s64(seed, stream)
     done = 0
     while done < count:
         c = min(chunk, count - done)
         i = torch.arange(start + done, start + done + c, dtype=torch.int64, device=device)
-        x = i * _s64(_ODD) + key
-        x = x ^ lsr(x, 30)
-        x = x * _s64(_M1)
-        x = x ^ lsr(x, 27)
-        x = x * _s64(_M2)
-        x = x ^ lsr(x, 31)
-        out[done : done + c] = q[lsr(x, 48)]
+        out[done : done + c] = fill_torch_at(key, i, q)
         done += c
     return out
