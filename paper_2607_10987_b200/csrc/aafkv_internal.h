@@ -101,6 +101,12 @@ struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
     int n;
     int total;
 };
+// Small batches travel as kernel parameters instead of through the pinned argument ring: the kernel then starts
+// without a read across PCIe and the host records no event for the ring slot.
+constexpr int SMALL_ARGS = 16;
+struct SmallInts {        // fork: children[k]; evict: ctx[n] followed by ent_off[n + 1]
+    int v[2 * SMALL_ARGS + 1];
+};
 
 // ---- launchers (each returns cudaGetLastError() of its launches)
 // `clock` is the logical clock of the call (count of successful state-touching calls); planners stamp
@@ -109,14 +115,16 @@ cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, l
                                     long long clock, cudaStream_t st, int table_j0 = 0);
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
                                long long clock, cudaStream_t st);
+// children_dev == nullptr: the k <= SMALL_ARGS children are in `small`
 cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
-                        long long clock, cudaStream_t st);
+                        const SmallInts &small, long long clock, cudaStream_t st);
 cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
                                int total_slots, int max_batch, int dry_run, long long clock, cudaStream_t st);
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
                                 int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st);
-cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
-                         long long clock, int *n_launches, cudaStream_t st);
+// args_dev == nullptr: the n <= SMALL_ARGS contexts and their entry offsets are in `small` (total <= 32768)
+cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,
+                         int total, long long clock, int *n_launches, cudaStream_t st);
 // Scored eviction (Alg. KV-Evict): result[0] = number of victims, result[1] = free blocks afterwards,
 // result[2..] = victims in eviction order; `result` is host memory the device can write.
 cudaError_t launch_evict_to_budget(const Geom &g, const DevState &s, double alpha, double beta, double gamma,

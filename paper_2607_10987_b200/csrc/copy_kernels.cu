@@ -73,8 +73,12 @@ __device__ __forceinline__ Unit decode_unit(const Piece *__restrict__ pieces, lo
     return r;
 }
 
-// Ticket counter of the dynamic work distribution (see the header comment).
-__device__ __forceinline__ long long take_ticket(DevCtl *ctl) { return (long long)atomicAdd(&ctl->copy_ticket, 1ull); }
+// Ticket counter of the dynamic work distribution (see the header comment).  Every drawer (a CTA of the bulk
+// engine, a warp of the warp engine) starts with the unit of its own index, so that the first loads of a launch do
+// not wait for an atomic; tickets number the units behind those, hence `first` = number of drawers.
+__device__ __forceinline__ long long take_ticket(DevCtl *ctl, long long first) {
+    return first + (long long)atomicAdd(&ctl->copy_ticket, 1ull);
+}
 // Called once per CTA when it has drawn its last ticket: the last CTA of the grid re-arms the counters.
 __device__ __forceinline__ void leave_copy(DevCtl *ctl) {
     __threadfence();
@@ -135,10 +139,10 @@ __global__ void __launch_bounds__(VEC_THREADS) copy_warp_kernel(const Piece *__r
     const long long total = (long long)n_slots * n_planes * cpp;
     const long long groups = (total + 31) / 32;  // a ticket is worth 32 consecutive units
     const int lane = threadIdx.x & 31;
-    long long grp = lane == 0 ? take_ticket(ctl) : 0;
-    grp = __shfl_sync(FULL, grp, 0);
+    const long long n_warps = (long long)gridDim.x * (VEC_THREADS / 32);
+    long long grp = (long long)blockIdx.x * (VEC_THREADS / 32) + (threadIdx.x >> 5);
     while (grp < groups) {
-        long long grp_next = lane == 0 ? take_ticket(ctl) : 0;  // drawn early: its latency hides behind the copies
+        long long grp_next = lane == 0 ? take_ticket(ctl, n_warps) : 0;  // drawn early: its latency hides behind the copies
         const long long base = grp * 32;
         Unit mine;
         mine.src = nullptr; mine.src2 = nullptr; mine.dst = nullptr; mine.nbytes = 0; mine.nbytes2 = 0;
@@ -223,7 +227,7 @@ cudaError_t launch_expire_wait(const DevState &s, long long limit_cycles, cudaSt
     return cudaGetLastError();
 }
 // L2 policy for data that is touched once: mark the lines evict-first so that the stream does not push
-// other tenants' data out of the 126 MB L2
+// other tenants' data out of the 126 MB L2 (optional: see copy_tuning_init)
 __device__ __forceinline__ unsigned long long l2_evict_first_policy() {
     unsigned long long pol;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
-    long long u_next = take_ticket(ctl);  // next unit to look at for loading
+    long long u_next = blockIdx.x;  // next unit to look at for loading
     int k_load = 0;                       // units whose load has been issued
     int k_store = 0;                      // units whose store has been issued
     bool timed_out = false;
@@ -284,7 +288,7 @@ __global__ void __launch_bounds__(32) copy_bulk_kernel(const Piece *__restrict__
     auto issue_load = [&]() -> bool {
         while (u_next < total) {
             const Unit un = decode_unit(pieces, u_next, n_slots, plane0, cpp, chunk);
-            u_next = take_ticket(ctl);
+            u_next = take_ticket(ctl, gridDim.x);
             const unsigned nb = un.nbytes + un.nbytes2;
             if (nb == 0) continue;
             const int s = k_load % stages;
@@ -365,7 +369,9 @@ cudaError_t copy_tuning_init(long long run, CopyTuning *t) {
     if (ctas < 1) ctas = 1;
     if (ctas > 8) ctas = 8;
     t->bulk_ctas = env_int("AAFKV_BULK_CTAS", ctas, 1, 16);
-    t->bulk_l2 = env_int("AAFKV_BULK_L2", 3, 0, 3);
+    // L2 evict-first hints (bit 0 loads, bit 1 stores) keep the stream from displacing other tenants' lines but cost
+    // about 1.5 % of the copy rate when the GPU runs nothing else: off unless asked for
+    t->bulk_l2 = env_int("AAFKV_BULK_L2", 0, 0, 3);
     t->vec_unroll = env_int("AAFKV_VEC_UNROLL", 4, 1, 8);
     if (t->vec_unroll == 3 || (t->vec_unroll > 4 && t->vec_unroll < 8)) t->vec_unroll = 4;
     t->warp_unroll = env_int("AAFKV_WARP_UNROLL", 8, 4, 8) == 4 ? 4 : 8;

@@ -191,10 +191,18 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevSt
 // ------------------------------------------------------------------------------------------
 // fork: k table copies, refcount += k per parent entry
 __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int parent, long long T, int k,
-                                                   const int *__restrict__ children_host, long long clock) {
+                                                   const int *__restrict__ children_host, SmallInts small,
+                                                   long long clock) {
     const int nblk = (int)((T + g.BS - 1) / g.BS);
     __shared__ int sh_children[1024];
-    const int *children = stage_args(children_host, k, sh_children, 1024);
+    const int *children;
+    if (children_host) {
+        children = stage_args(children_host, k, sh_children, 1024);
+    } else {  // a small fan-out arrives as kernel parameters
+        if (threadIdx.x < k) sh_children[threadIdx.x] = small.v[threadIdx.x];
+        __syncthreads();
+        children = sh_children;
+    }
     const int *pt = s.tables + (long long)parent * g.max_blk;
     const long long total = (long long)nblk * k;
     for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
@@ -597,10 +605,17 @@ __global__ void __launch_bounds__(256) evict_release_kernel(Geom g, DevState s, 
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS) evict_fused_kernel(Geom g, DevState s,
-                                                                   const EvictArgs *__restrict__ a, int n, int total,
-                                                                   unsigned long long stamp) {
+                                                                   const EvictArgs *__restrict__ a, SmallInts small,
+                                                                   int n, int total, unsigned long long stamp) {
     __shared__ int sh_args[EVICT_STAGE];
-    const int *ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    const int *ctx;
+    if (a) {
+        ctx = stage_args(reinterpret_cast<const int *>(a + 1), 2 * n + 1, sh_args, EVICT_STAGE);
+    } else {  // a small batch arrives as kernel parameters
+        if (threadIdx.x < 2 * n + 1) sh_args[threadIdx.x] = small.v[threadIdx.x];
+        __syncthreads();
+        ctx = sh_args;
+    }
     const int *ent_off = ctx + n;
     for (int e = threadIdx.x; e < total; e += blockDim.x) evict_release_entry(g, s, ctx, ent_off, n, e, stamp);
     __syncthreads();  // one CTA: every reference has been dropped and every mark set
@@ -782,9 +797,9 @@ cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long l
     return cudaGetLastError();
 }
 cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
-                        long long clock, cudaStream_t st) {
+                        const SmallInts &small, long long clock, cudaStream_t st) {
     const long long nblk = (T + g.BS - 1) / g.BS;
-    fork_kernel<<<grid_for(nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, T, k, children_dev, clock);
+    fork_kernel<<<grid_for(nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, T, k, children_dev, small, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
@@ -798,14 +813,15 @@ cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeS
                                                     clock);
     return cudaGetLastError();
 }
-cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, int n, int total,
-                         long long clock, int *n_launches, cudaStream_t st) {
+cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,
+                         int total, long long clock, int *n_launches, cudaStream_t st) {
     const unsigned long long stamp = (unsigned long long)clock << 32;
     if (total <= EVICT_FUSED_MAX) {
         *n_launches = 1;
-        evict_fused_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, n, total, stamp);
+        evict_fused_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, args_dev, small, n, total, stamp);
         return cudaGetLastError();
     }
+    if (!args_dev) return cudaErrorInvalidValue;  // the grid path reads its records from memory
     *n_launches = 4;
     const int n_tiles = (total + EVICT_TILE - 1) / EVICT_TILE;
     evict_release_kernel<<<grid_for(total, 256, 148), 256, 0, st>>>(g, s, args_dev, n, total, stamp);

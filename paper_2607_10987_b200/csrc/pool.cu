@@ -667,15 +667,19 @@ int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_chil
     DeviceGuard guard(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
-    int *children = reinterpret_cast<int *>(acquire_args(p));
+    // a small fan-out travels as kernel parameters, a large one through the pinned argument ring
+    SmallInts small{};
+    const bool by_value = k <= SMALL_ARGS;
+    int *children = by_value ? small.v : reinterpret_cast<int *>(acquire_args(p));
     int c = -1;
     for (int j = 0; j < k; ++j) {
         c = smallest_free_ctx(p, c + 1);
         children[j] = c;
     }
     const long long T = p->len[parent];
-    const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, children, p->clock + 1, p->meta_stream);
-    release_args(p, p->meta_stream);
+    const cudaError_t e = launch_fork(p->g, p->s, parent, T, k, by_value ? nullptr : children, small, p->clock + 1,
+                                      p->meta_stream);
+    if (!by_value) release_args(p, p->meta_stream);
     if (e != cudaSuccess) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
@@ -890,21 +894,28 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
     DeviceGuard guard(p->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
-    EvictArgs *a = reinterpret_cast<EvictArgs *>(acquire_args(p));
-    int *ctx = reinterpret_cast<int *>(a + 1);
-    int *ent_off = ctx + n;
     long long total = 0;
+    for (int i = 0; i < n; ++i) total += nblk_of(p, p->len[ctxs[i]]);
+    // a small batch travels as kernel parameters, a large one through the pinned argument ring
+    SmallInts small{};
+    const bool by_value = n <= SMALL_ARGS && total <= 32768;
+    EvictArgs *a = by_value ? nullptr : reinterpret_cast<EvictArgs *>(acquire_args(p));
+    int *ctx = by_value ? small.v : reinterpret_cast<int *>(a + 1);
+    int *ent_off = ctx + n;
+    total = 0;
     for (int i = 0; i < n; ++i) {
         ctx[i] = ctxs[i];
         ent_off[i] = (int)total;
         total += nblk_of(p, p->len[ctxs[i]]);
     }
     ent_off[n] = (int)total;
-    a->n = n;
-    a->total = (int)total;
+    if (a) {
+        a->n = n;
+        a->total = (int)total;
+    }
     int n_launches = 0;
-    const cudaError_t e = launch_evict(p->g, p->s, a, n, (int)total, p->clock + 1, &n_launches, p->meta_stream);
-    release_args(p, p->meta_stream);
+    const cudaError_t e = launch_evict(p->g, p->s, a, small, n, (int)total, p->clock + 1, &n_launches, p->meta_stream);
+    if (a) release_args(p, p->meta_stream);
     if (e != cudaSuccess) return broke(p);
     p->clock += 1;
     p->meta_launches += n_launches;
