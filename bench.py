@@ -379,6 +379,45 @@ def extra_report(args):
     elif args.workload == "compose":
         out["share"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=False)
         out["copy_all"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=True)
+    elif args.workload == "costmodel":
+        # Transfer time of the paper's largest state over its network grid (Sec. 5.4: |KV| / BW + delta; Exp. 3:
+        # 10-400 Gbps, 10 / 100 us), with the pack / unpack term measured here beside it, and the decision
+        # pi(S) = transfer iff T_transfer < T_prefill for a range of assumed prefill times (the paper's measured
+        # prefill times are not available).
+        g = configs.Geometry(32, 8, 128, 16, 2, 8192, 8, 4096)
+        seed, T = configs.SEED_BASE + 2, 32640
+        be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False,
+                        staging_tokens=T)
+        buf = be.payload(seed, 1, T)
+        acc = {"materialize": [0.0, 0], "import": [0.0, 0]}
+        for it in range(args.warmup + args.steps):
+            res = {}
+            _, dms, dl, _ = timed_ops(be.o, lambda: res.update(c=be.imp(buf, T)))
+            _, dms2, dl2, _ = timed_ops(be.o, lambda: res.update(m=be.materialize(res["c"][1], 0, T)))
+            assert res["c"][0] == 0 and res["m"][0] == 0
+            be.evict([res["c"][1]])
+            if it >= args.warmup:
+                acc["import"][0] += dms["import"]; acc["import"][1] += dl["import"]
+                acc["materialize"][0] += dms2["materialize"]; acc["materialize"][1] += dl2["materialize"]
+        kv = binding.aaf_kv_state_bytes(g.n_layers, g.n_kv_heads, g.head_dim, g.elt_bytes, T)
+        pack = 2 * kv * acc["materialize"][1] / (acc["materialize"][0] * 1e-3)   # bytes read + written per second
+        unpack = 2 * kv * acc["import"][1] / (acc["import"][0] * 1e-3)
+        rate = 2.0 / (1.0 / pack + 1.0 / unpack)  # one rate for pack and unpack together
+        rows = []
+        links = [(f"{gb} Gbps", gb * 1e9 / 8) for gb in (10, 25, 100, 200, 400)] + [("NVLink 5, 900 GB/s", 900e9)]
+        for name, bw in links:
+            for lat in (10e-6, 100e-6):
+                wire = binding.aaf_kv_transfer_time(kv, bw, lat)
+                full = binding.aaf_kv_transfer_time_packed(kv, bw, lat, rate)
+                rows.append({"link": name, "latency_us": lat * 1e6, "T_transfer_ms": wire * 1e3,
+                             "T_with_pack_unpack_ms": full * 1e3, "pack_unpack_share": (full - wire) / full,
+                             "transfer_wins_if_prefill_exceeds_ms": full * 1e3,
+                             "policy_at_prefill_1s": binding.aaf_kv_policy(False, full, 1.0),
+                             "policy_at_prefill_100ms": binding.aaf_kv_policy(False, full, 0.1)})
+        out.update({"state_tokens": T, "state_bytes": kv, "pack_GBps_read_plus_written": pack / 1e9,
+                    "unpack_GBps_read_plus_written": unpack / 1e9, "pack_ms": 2 * kv / pack * 1e3,
+                    "unpack_ms": 2 * kv / unpack * 1e3, "policy_codes": {"reuse": 0, "transfer": 1, "recompute": 2},
+                    "rows": rows})
     elif args.workload == "meta":
         # metadata-only operators: rate of back-to-back calls (host launch + device execution), against the
         # rate of back-to-back launches of a trivial kernel on the same stream (the launch floor)

@@ -317,6 +317,31 @@ int aaf_kv_sync_status(aaf_kv_pool *pool);
 int aaf_kv_set_copy_engine(aaf_kv_pool *pool, int engine);  /* AAF_ENGINE_* */
 int aaf_kv_set_timing(aaf_kv_pool *pool, int enable);       /* bracket copy kernels with CUDA events */
 
+/* Cost model of the state path (host-only arithmetic; no device is touched, no pool is needed).
+ *   aaf_kv_state_bytes   |KV| of n_tokens tokens: n_tokens * 2 * n_layers * n_kv_heads * head_dim * elt_bytes
+ *                        (K and V blocks of every layer, Sec. 3.2); -1 if an argument is not positive or the
+ *                        product overflows.
+ *   aaf_kv_transfer_time T_transfer = |KV| / BW + delta (Sec. 5.4; Exp. 3: KV bytes / bandwidth + latency),
+ *                        evaluated in double precision as one division and one addition, in that order.
+ *                        Returns a NaN for kv_bytes < 0, bandwidth <= 0 or latency < 0.
+ *   aaf_kv_transfer_time_packed  the same plus the term the paper's model leaves out: packing the state into
+ *                        a transfer buffer at the sender and unpacking it at the receiver (aaf_kv_materialize /
+ *                        aaf_kv_import), each moving 2 |KV| bytes (read + written) at pack_rate bytes per second
+ *                        (read + written, as the library's benchmark reports it):
+ *                        T = 2 |KV| / pack_rate + (|KV| / BW + delta) + 2 |KV| / pack_rate, summed left to right.
+ *                        This is the un-overlapped upper bound; the chunked forms overlap packing with the wire.
+ *   aaf_kv_policy        the scheduling rule pi(S) (Sec. 4.6; App. C; App. E step 5): AAF_POLICY_REUSE if the
+ *                        state is local and compatible, else AAF_POLICY_TRANSFER iff t_transfer < t_prefill
+ *                        (strictly), else AAF_POLICY_RECOMPUTE.  A NaN time compares false: recompute. */
+#define AAF_POLICY_REUSE 0
+#define AAF_POLICY_TRANSFER 1
+#define AAF_POLICY_RECOMPUTE 2
+int64_t aaf_kv_state_bytes(int32_t n_layers, int32_t n_kv_heads, int32_t head_dim, int32_t elt_bytes, int64_t n_tokens);
+double aaf_kv_transfer_time(double kv_bytes, double bandwidth_bytes_per_s, double latency_s);
+double aaf_kv_transfer_time_packed(double kv_bytes, double bandwidth_bytes_per_s, double latency_s,
+                                   double pack_rate_bytes_per_s);
+int aaf_kv_policy(int local_and_compatible, double t_transfer_s, double t_prefill_s);
+
 /* Gather for callers that cannot allocate -- the paper has no counterpart; this is a library
  * convenience.  Same result as aaf_kv_materialize (dst[l][kv][t - tok_begin] =
  * pool[l][table[t / BS]][kv][t % BS] for t in [tok_begin, tok_end)), but it needs no pool object and

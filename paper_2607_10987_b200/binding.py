@@ -21,6 +21,7 @@ AAF_ERR_TOO_LONG, AAF_ERR_INCOMPAT, AAF_ERR_DST_TOO_SMALL, AAF_ERR_CUDA = -5, -6
 AAF_ERR_CORRUPT, AAF_ERR_TIMEOUT, AAF_ERR_TOO_MANY, AAF_ERR_SCRATCH_LIMIT = -9, -10, -11, -12
 AAF_NOALLOC_MAX_BLOCKS = 4096
 AAF_COMPOSE_SHARE, AAF_COMPOSE_COPY_ALL = 0, 1
+AAF_POLICY_REUSE, AAF_POLICY_TRANSFER, AAF_POLICY_RECOMPUTE = 0, 1, 2
 AAF_ENGINE_AUTO, AAF_ENGINE_VEC, AAF_ENGINE_BULK, AAF_ENGINE_WARP = 0, 1, 2, 3
 AAF_OP_MATERIALIZE, AAF_OP_IMPORT, AAF_OP_APPEND, AAF_OP_COMPOSE, AAF_OP_CLASSES = 0, 1, 2, 3, 4
 OP_NAMES = ("materialize", "import", "append", "compose")
@@ -96,6 +97,10 @@ SYMBOLS = {
     "aaf_kv_set_timing": (C.c_int, [_vp, C.c_int]),
     "aaf_kv_materialize_noalloc": (C.c_int, [_vp, _sz, _i32, _i32, _i32, _i32, _i32, _i32, _p32, _i32, _i64, _i64, _vp,
                                              _sz, _vp]),
+    "aaf_kv_state_bytes": (C.c_int64, [_i32, _i32, _i32, _i32, _i64]),
+    "aaf_kv_transfer_time": (C.c_double, [C.c_double, C.c_double, C.c_double]),
+    "aaf_kv_transfer_time_packed": (C.c_double, [C.c_double, C.c_double, C.c_double, C.c_double]),
+    "aaf_kv_policy": (C.c_int, [C.c_int, C.c_double, C.c_double]),
     "aaf_kv_debug_expire_wait": (C.c_int, [_vp, C.c_uint64, _vp]),
     "aaf_kv_strerror": (C.c_char_p, [C.c_int]),
 }
@@ -167,6 +172,13 @@ def aaf_kv_materialize_noalloc(pool_base, layer_stride, n_layers, n_kv_heads, he
     return _fn("aaf_kv_materialize_noalloc")(pool_base, layer_stride, n_layers, n_kv_heads, head_dim, block_size,
                                              elt_bytes, n_blocks, block_table_host, n_table_blocks, t0, t1, dst,
                                              dst_bytes, stream)
+def aaf_kv_state_bytes(n_layers, n_kv_heads, head_dim, elt_bytes, n_tokens):
+    return _fn("aaf_kv_state_bytes")(n_layers, n_kv_heads, head_dim, elt_bytes, n_tokens)
+def aaf_kv_transfer_time(kv_bytes, bandwidth, latency): return _fn("aaf_kv_transfer_time")(kv_bytes, bandwidth, latency)
+def aaf_kv_transfer_time_packed(kv_bytes, bandwidth, latency, pack_rate):
+    return _fn("aaf_kv_transfer_time_packed")(kv_bytes, bandwidth, latency, pack_rate)
+def aaf_kv_policy(local_and_compatible, t_transfer, t_prefill):
+    return _fn("aaf_kv_policy")(1 if local_and_compatible else 0, t_transfer, t_prefill)
 def aaf_kv_debug_expire_wait(pool, limit_cycles, stream): return _fn("aaf_kv_debug_expire_wait")(pool, limit_cycles, stream)
 def aaf_kv_strerror(status): return _fn("aaf_kv_strerror")(status).decode()
 
