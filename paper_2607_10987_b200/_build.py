@@ -29,6 +29,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
                "-Xcompiler", "-fPIC", "-shared", "-I", INCLUDE, "-I", CSRC, "-o", LIB] + sources()
+        if os.environ.get("AAFKV_NVTX"):  # profiler ranges around every C-ABI operator call
+            cmd.insert(1, "-DAAFKV_NVTX")
+            cmd += ["-ldl"]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

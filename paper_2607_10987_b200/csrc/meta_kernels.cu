@@ -250,14 +250,22 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
         tailb[i] = r > 0 ? s.tables[(long long)ent[i].ctx * g.max_blk + (T - 1) / g.BS] : -1;
     }
     __syncthreads();
-    // phase 2: copy-on-write decision and block need of every entry
+    // phase 2: copy-on-write decision and block need of every entry.  The rank of an entry among the earlier
+    // entries with the same tail block is a scan of tailb[0 .. i): from shared memory when the batch fits.
+    __shared__ int sh_tailb[1024];
+    const int *tb = tailb;
+    if (n <= 1024) {
+        for (int i = threadIdx.x; i < n; i += blockDim.x) sh_tailb[i] = tailb[i];
+        __syncthreads();
+        tb = sh_tailb;
+    }
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const long long T = ent[i].T;
-        const int b = tailb[i];
+        const int b = tb[i];
         int cow = 0;
         if (b >= 0) {
             int rank = 0;
-            for (int i2 = 0; i2 < i; ++i2) rank += (tailb[i2] == b);
+            for (int i2 = 0; i2 < i; ++i2) rank += (tb[i2] == b);
             cow = rank < s.refcount[b] - 1;
         }
         const int fresh = (int)((T + ent[i].n_new + g.BS - 1) / g.BS - (T + g.BS - 1) / g.BS);

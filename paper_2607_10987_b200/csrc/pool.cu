@@ -20,6 +20,21 @@
 
 #include "aafkv_internal.h"
 
+// Profiler ranges: built with -DAAFKV_NVTX every C-ABI operator call is an NVTX range named after the entry
+// point (header-only NVTX 3, no extra library); without the switch the macro is empty.
+#ifdef AAFKV_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace {
+struct ScopedRange {
+    explicit ScopedRange(const char *name) { nvtxRangePushA(name); }
+    ~ScopedRange() { nvtxRangePop(); }
+};
+}  // namespace
+#define AAF_RANGE(name) ScopedRange aaf_range_(name)
+#else
+#define AAF_RANGE(name) do { } while (0)
+#endif
+
 using namespace aafkv;
 
 namespace {
@@ -380,6 +395,7 @@ size_t aaf_kv_pool_workspace_bytes(const aaf_kv_pool_desc *desc) {
 }
 
 int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
+    AAF_RANGE("aaf_kv_pool_create");
     if (!out) return AAF_ERR_INVALID_ARG;
     *out = nullptr;
     if (!geometry_ok(desc)) return AAF_ERR_INVALID_ARG;
@@ -507,6 +523,7 @@ int aaf_kv_pool_destroy(aaf_kv_pool *p) {
 
 int aaf_kv_materialize(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_dev,
                        size_t dst_bytes, aaf_kv_xfer_desc *out_desc, void *stream) {
+    AAF_RANGE("aaf_kv_materialize");
     if (!p) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
@@ -517,6 +534,7 @@ int aaf_kv_materialize(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t
 int aaf_kv_materialize_host(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, int64_t tok_end, void *dst_host,
                             size_t dst_bytes, void *staging_dev, size_t staging_bytes, aaf_kv_xfer_desc *out_desc,
                             void *stream) {
+    AAF_RANGE("aaf_kv_materialize_host");
     if (!p || !dst_host) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
@@ -533,6 +551,7 @@ int aaf_kv_materialize_host(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t tok_begin, in
 
 int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
                   void *stream) {
+    AAF_RANGE("aaf_kv_import");
     if (!p) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
@@ -541,6 +560,7 @@ int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *d
 
 int aaf_kv_import_host(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
                        size_t staging_bytes, aaf_ctx_t *out_ctx, void *stream) {
+    AAF_RANGE("aaf_kv_import_host");
     if (!p || !src_host || !desc) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
@@ -553,6 +573,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
                                     size_t dst_bytes, void *staging_dev, size_t staging_bytes, int32_t chunk_tokens,
                                     uint32_t *done_flags_host, int32_t flags_cap, int32_t *n_chunks_out,
                                     aaf_kv_xfer_desc *out_desc, void *stream) {
+    AAF_RANGE("aaf_kv_materialize_host_chunked");
     if (!p || !dst_host || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     if (!is_live(p, ctx)) return AAF_ERR_BAD_CTX;
@@ -606,6 +627,7 @@ int aaf_kv_materialize_host_chunked(aaf_kv_pool *p, aaf_ctx_t ctx, int64_t t0, i
 
 int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,
                                size_t staging_bytes, int32_t chunk_tokens, aaf_ctx_t *out_ctx, void *stream) {
+    AAF_RANGE("aaf_kv_import_host_chunked");
     if (!p || !src_host || !desc || !out_ctx || chunk_tokens < 1 || chunk_tokens % p->g.BS != 0 ||
         !aligned16(staging_dev))
         return AAF_ERR_INVALID_ARG;
@@ -659,6 +681,7 @@ int aaf_kv_import_host_chunked(aaf_kv_pool *p, const void *src_host, const aaf_k
 }
 
 int aaf_kv_fork(aaf_kv_pool *p, aaf_ctx_t parent, int32_t k, aaf_ctx_t *out_children, void *stream) {
+    AAF_RANGE("aaf_kv_fork");
     if (!p || !out_children || k < 1) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     if (!is_live(p, parent)) return AAF_ERR_BAD_CTX;
@@ -708,6 +731,7 @@ static int append_check(const aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, 
 
 int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
                   const void *const *src_dev, void *stream) {
+    AAF_RANGE("aaf_kv_append");
     if (!p || n < 1 || !ctxs || !n_new || !src_dev) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     {
@@ -779,6 +803,7 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
 
 int aaf_kv_append_host(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_t *n_new,
                        const void *const *src_host, void *staging_dev, size_t staging_bytes, void *stream) {
+    AAF_RANGE("aaf_kv_append_host");
     if (!p || n < 1 || !ctxs || !n_new || !src_host || !aligned16(staging_dev)) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     {
@@ -819,6 +844,7 @@ int aaf_kv_append_host(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const i
 
 int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
                    void *stream) {
+    AAF_RANGE("aaf_kv_compose");
     if (!p || m < 1 || !segs || !out_ctx || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     if (m > p->lay.max_batch) return AAF_ERR_TOO_MANY;
@@ -881,6 +907,7 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
 }
 
 int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {
+    AAF_RANGE("aaf_kv_evict");
     if (!p || n < 1 || !ctxs) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
@@ -926,6 +953,7 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
 
 int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gamma, int64_t budget_blocks,
                            aaf_ctx_t *out_victims, int32_t cap, int32_t *n_victims, void *stream) {
+    AAF_RANGE("aaf_kv_evict_to_budget");
     if (!p || !out_victims || !n_victims || budget_blocks < 0) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     if (!(alpha == alpha && beta == beta && gamma == gamma) || alpha - alpha != 0.0 || beta - beta != 0.0 ||
@@ -965,6 +993,7 @@ int aaf_kv_catalog_rows(aaf_kv_pool *p, int32_t *n_states, int64_t *n_block_rows
 }
 
 int aaf_kv_export_catalog(aaf_kv_pool *p, const aaf_kv_catalog_cols *cols, void *stream) {
+    AAF_RANGE("aaf_kv_export_catalog");
     if (!p || !cols) return AAF_ERR_INVALID_ARG;
     if (p->broken) return AAF_ERR_CUDA;
     int32_t ns = 0;
