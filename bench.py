@@ -698,8 +698,8 @@ def measure_step(w, args, cl, dev_index, steps, warmup, min_seconds, clocks_for_
         h2d, d2h = (T + agents * n_new) * g.bpt, T * g.bpt
 
         # what PCIe allows for this step: plain copies of the same pinned buffers, each direction alone and both at
-        # once (the directions slow each other down).  The step must upload h2d bytes and download d2h bytes; the
-        # download can only overlap the upload of the continuation tokens.
+        # once (the directions slow each other down).  A step must upload h2d bytes and download d2h bytes; in
+        # steady state the download of one step overlaps uploads of the same and the next step.
         def copy_ms(pairs):
             evs = []
             torch.cuda.synchronize()

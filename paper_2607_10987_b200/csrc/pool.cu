@@ -948,7 +948,14 @@ int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream)
     p->meta_launches += n_launches;
     for (int i = 0; i < n; ++i) p->len[ctxs[i]] = -1;
     p->live_ctx -= n;
-    return AAF_OK;  // the lower bound of the free count stays valid: evict only adds free blocks
+    // The lower bound of the free count stays valid (evict only adds free blocks), and the host can raise it without
+    // asking the device: a live block is named by at least one table entry, so at most sum(table lengths) blocks
+    // are live.  A caller that evicts what it created therefore never pays the synchronising refresh.
+    long long entries = 0;
+    for (int c = 0; c < p->g.max_ctx; ++c)
+        if (p->len[c] >= 0) entries += nblk_of(p, p->len[c]);
+    p->free_lb = std::max(p->free_lb, (long long)p->g.NB - entries);
+    return AAF_OK;
 }
 
 int aaf_kv_evict_to_budget(aaf_kv_pool *p, double alpha, double beta, double gamma, int64_t budget_blocks,
