@@ -34,7 +34,9 @@
  * library allocates host memory only (the pool object, a pinned argument ring, events).
  *
  * Ordering: calls on one pool are applied in call order and must be issued to one stream
- * (or the caller orders streams itself).  Data calls are asynchronous.  Every kernel that
+ * (or the caller orders streams itself; the library additionally makes the copy launches of a pool
+ * run one after the other when consecutive calls name different streams, because they share a work
+ * counter in the pool's control block).  Data calls are asynchronous.  Every kernel that
  * touches payload bytes (pool rows, transfer buffers) runs on the `stream` argument, so the
  * caller's own work on that stream is ordered against them as usual.  Kernels that touch only
  * the library's metadata (block tables, reference counts, the ring, copy descriptors) run on a

@@ -123,6 +123,11 @@ struct aaf_kv_pool {
     cudaStream_t meta_stream = nullptr;
     cudaEvent_t plan_done[2] = {}, copy_done[2] = {};
     int next_buf = 0;
+    // Copy launches of a pool share the ticket counter of its control block, so they must never overlap on the
+    // device.  Calls on one stream are ordered anyway; when a call arrives on ANOTHER stream than the previous
+    // copy launch, that stream is made to wait for the previous operator's last copy launch first.
+    cudaStream_t last_copy_stream = nullptr;
+    cudaEvent_t last_copy_event = nullptr;
     // pinned argument ring
     char *args = nullptr;
     size_t slot_bytes = 0;
@@ -252,6 +257,8 @@ bool end_plan(aaf_kv_pool *p, const PlanSlot &ps, cudaStream_t st) {
 // After the operator's last copy launch: mark the buffer's readers done and switch buffers.
 void end_copy(aaf_kv_pool *p, const PlanSlot &ps, cudaStream_t st) {
     cudaEventRecord(p->copy_done[ps.buf], st);
+    p->last_copy_stream = st;
+    p->last_copy_event = p->copy_done[ps.buf];
     p->next_buf ^= 1;
 }
 
@@ -262,6 +269,10 @@ int run_copy(aaf_kv_pool *p, const PlanSlot &ps, int cls, int n_slots, long long
     view.pieces += piece0;  // a launch may cover a sub-range of the planned pieces (chunked transfers)
     const long long avg_piece = n_slots > 0 ? payload_tokens * p->g.row / n_slots : 0;
     if (n_slots <= 0) return AAF_OK;
+    if (p->last_copy_event && st != p->last_copy_stream) {  // a different stream: serialise behind the last copy launch
+        if (cudaStreamWaitEvent(st, p->last_copy_event, 0) != cudaSuccess) return AAF_ERR_CUDA;
+        p->last_copy_stream = st;  // the wait is queued; later launches of this operator need not repeat it
+    }
     TimedLaunch t{};
     if (p->timing) {
         t.start = get_event(p);

@@ -212,6 +212,30 @@ def test_chunked_host_transfer_is_byte_identical_and_flags_every_chunk(chunk_tok
     assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
 
 
+def test_calls_on_alternating_streams_do_not_overlap_their_copy_launches():
+    """Data-independent operators of one pool issued to two streams without any ordering by the caller: the
+    library serialises their copy launches (they share the pool's work counter), so every byte still arrives."""
+    g = Geometry(4, 8, 128, 16, 2, 1024, 32, 64)  # 2 KiB rows, 32 KiB runs: the bulk engine
+    order = configs.free_order(SEED, g.n_blocks)
+    gpu = GpuBackend(g, SEED, free_order=order, init_fill=False)
+    cpu = OracleBackend(g, SEED, free_order=order, init_fill=False)
+    gpu.o.pool.zero_()
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(gpu.o.device), torch.cuda.Stream(gpu.o.device)]
+    lens = [600 + 37 * i for i in range(12)]
+    bufs = [gpu.payload(SEED, 1 + i, n) for i, n in enumerate(lens)]
+    torch.cuda.synchronize()
+    for i, n in enumerate(lens):
+        with torch.cuda.stream(streams[i % 2]):
+            st, c = gpu.imp(bufs[i], n)
+        assert (st, c) == (0, i)
+        assert cpu.imp(cpu.payload(SEED, 1 + i, n), n) == (0, i)
+    torch.cuda.synchronize()
+    assert gpu.snapshot() == cpu.snapshot()
+    assert np.array_equal(gpu.pool_layers(range(g.n_layers)), cpu.o.pool_view())
+    assert gpu.o.sync_status() == 0
+
+
 def test_two_pools_of_different_geometry_interleaved():
     """Launch shapes and scratch are per pool: two pools with different rows, block sizes and engines,
     used alternately on the same stream, each stay bit-exact against their own oracle."""

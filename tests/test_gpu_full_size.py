@@ -138,6 +138,60 @@ def test_config3_compose_levels_value_model_all_layers(copy_all):
     assert sh.vm.ctx[max(sh.vm.ctx)] == sh.vm.ctx[max(sh.vm.ctx) - 1] and len(sh.vm.ctx[max(sh.vm.ctx)]) == sum(lens)
 
 
+def test_config2_host_buffer_path_value_model_all_layers():
+    """The end-to-end form of the 8B step, as the benchmark times it: every input arrives from pinned host memory
+    through the library's host-buffer calls (chunked import, chunked materialize, append from host buffers), on
+    the full 64 GiB pool.  The bytes that come back to the host and every live context (all layers) are compared
+    with what the value model says they must be."""
+    import torch
+
+    from tests.value_check import Paired
+
+    g, seed, _ = configs.config2(True)
+    if not _fits(g, 12):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    T, agents, n_new = 8187, 16, 512
+    gpu = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), init_fill=False)
+    sh = ShadowBackend(gpu)
+    pool, dev = gpu.o, gpu.o.device
+    root = sh.payload(seed, 1, T)
+    conts = [sh.payload(seed, 2 + i, n_new) for i in range(agents)]
+    h_root = torch.empty(T * g.bpt, dtype=torch.uint8).pin_memory()
+    h_root.copy_(root.dev)
+    h_conts = [torch.empty(n_new * g.bpt, dtype=torch.uint8).pin_memory() for _ in conts]
+    for h, c in zip(h_conts, conts):
+        h.copy_(c.dev)
+    h_out = torch.zeros(T * g.bpt, dtype=torch.uint8).pin_memory()
+    d_root = torch.empty(T * g.bpt, dtype=torch.uint8, device=dev)
+    d_conts = torch.empty(agents * n_new * g.bpt, dtype=torch.uint8, device=dev)
+    staging = torch.empty(T * g.bpt, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    for rnd in range(2):  # twice: the second round reuses every staging buffer while the first is still in flight
+        st, c_root = pool.import_host_chunked(h_root, T, d_root, 1024)
+        assert st == 0 and sh.vm.imp(root.tokens) == c_root
+        st, _ = pool.materialize_host_chunked(c_root, 0, T, h_out, staging, 1024)
+        assert st == 0
+        st, c_recv = pool.imp(staging, T)
+        assert st == 0 and sh.vm.imp(sh.vm.materialize(c_root, 0, T)) == c_recv
+        st, kids = pool.fork(c_recv, agents)
+        assert st == 0 and sh.vm.fork(c_recv, agents) == kids
+        assert pool.append_host(kids, [n_new] * agents, h_conts, d_conts) == 0
+        for k, c in zip(kids, conts):
+            sh.vm.append(k, c.tokens)
+        st, merged = pool.compose(kids[:2], 0)
+        assert st == 0 and sh.vm.compose(kids[:2]) == merged
+        if rnd == 0:
+            everything = [c_root, c_recv] + kids + [merged]
+            assert pool.evict(everything)[0] == 0
+            sh.vm.evict(everything)
+    torch.cuda.synchronize()
+    assert torch.equal(h_out, h_root)
+    sh.check_buffer(seed, Paired(h_out.to(dev), root.tokens))
+    sh.check_all_live(seed)
+    check_conservation(gpu.snapshot(), g.n_blocks, g.block_size)
+    assert pool.sync_status() == 0 and pool.stats()["cow_count"] == 2 * agents
+
+
 def test_config4_llama70b_value_model_all_layers():
     g, seed, ops = configs.config4(True)
     if not _fits(g, 40):
