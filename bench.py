@@ -79,6 +79,17 @@ def workload(name: str):
     raise SystemExit(f"unknown workload {name}")
 
 
+def step_config(w, n_blocks, engine):
+    """`config` of the JSON line: the same dict on both arms (the closed-form byte count needs no device)."""
+    g = w["g"]
+    moved = 2 * sum(class_tokens(g, w["T"], w["agents"], w["n_new"]).values()) * g.bpt
+    return {"workload": w["name"], "n_blocks": n_blocks, "pool_GiB": g.n_layers * n_blocks * 2 * g.run / 2**30,
+            "l2_policy": ("inputs_exceed_l2 (each operator streams %.1f GiB or more)" % (w["T"] * g.bpt / 2**30)
+                          if w["T"] * g.bpt > (256 << 20) else "none: smaller than the L2, a test shape, not a bench line"),
+            "parallelism": "replicas only",
+            "engine": engine, "moved_GB_per_step": moved / 1e9}
+
+
 def class_tokens(g, T, agents, n_new):
     """Tokens each operator class copies in one step (closed form of the step above)."""
     r = T % g.block_size
@@ -152,7 +163,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------- CPU oracle arm
-def oracle_rate(w, layers_sample: int, budget_s: float, max_steps: int):
+def oracle_rate(w, layers_sample: int, budget_s: float, max_steps: int, warm_steps: int = 1):
     """Times the CPU oracle, as it stands, on the same step restricted to `layers_sample` layers."""
     from oracle import paged
 
@@ -171,7 +182,8 @@ def oracle_rate(w, layers_sample: int, budget_s: float, max_steps: int):
         compose = staticmethod(lambda segs, fl: o.compose(segs, fl))
         materialize = staticmethod(lambda c, a, b: o.materialize(c, a, b))
 
-    step_ops(B, root, bufs, w["T"], w["agents"], w["n_new"], None)  # warm-up (page faults of the pool)
+    for _ in range(max(warm_steps, 1)):  # warm-up (page faults of the pool)
+        step_ops(B, root, bufs, w["T"], w["agents"], w["n_new"], None)
     rows0 = o.stats()["rows_copied"]
     t0 = time.perf_counter()
     steps = 0
@@ -189,14 +201,15 @@ def reference_arm(args, w):
         return
     layers = 2 if w["g"].n_layers > 2 else w["g"].n_layers
     # `steps` timed passes, each a bounded sample of the workload (a subset of the layers)
-    gbps, steps, dt, ops_s = oracle_rate(w, layers, budget_s=1e9, max_steps=max(args.steps, 1))
+    warm = max(args.warmup, 3)
+    gbps, steps, dt, ops_s = oracle_rate(w, layers, budget_s=1e9, max_steps=max(args.steps, 1), warm_steps=warm)
     cores = 1
     sample = f"{layers} of {w['g'].n_layers} layers of the step, {steps} passes, single thread"
     line = {
         "impl": "reference", "metric": METRIC, "value": gbps, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": 1, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": dt / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": w["name"], "sample": sample},
+        "config": step_config(w, w["g"].n_blocks, args.engine),
         "cpu_baseline": {"value": gbps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "ops_per_s": ops_s,
@@ -825,9 +838,7 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "repeats": r["repeats"], "timed_seconds": sum(r["region_ms"]) / 1e3,
-        "config": {"workload": w["name"], "n_blocks": r["n_blocks"], "pool_GiB": r["pool_GiB"],
-                   "l2_policy": "inputs_exceed_l2 (each operator streams >= 1 GiB)", "parallelism": "replicas only",
-                   "engine": args.engine, "moved_GB_per_step": r["moved_per_step"] / 1e9},
+        "config": step_config(w, r["n_blocks"], args.engine),
         "ops_per_s": world * 7 * total_steps / (sum(r["region_ms"]) * 1e-3),
         "gpu_launches": r["launches_per_region"],
         "clocks": r["clocks"], "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu_baseline,
