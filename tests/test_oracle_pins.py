@@ -74,6 +74,21 @@ def test_worked_example_w1():
     assert st == 0
     assert o.table(c1).tolist() == [int(x) for x in g["c1.table"].split()]
     assert np.array_equal(o.materialize(P, 0, 6)[1], enc([f"p{i}" for i in range(6)]))
+    # the merge policy that forbids aliasing, on a copy of the state: fresh blocks in increasing table position
+    oc = o.clone()
+    st, Zc = oc.compose([c1, c2], paged.COMPOSE_COPY_ALL)
+    assert (st, Zc) == (0, 3)
+    assert oc.table(Zc).tolist() == [int(x) for x in g["Zc.table"].split()]
+    pvc = oc.pool_view()
+    for key in ("Zc.block5", "Zc.block2", "Zc.block7", "Zc.block6"):
+        b = int(key[8:])
+        for s, tok in enumerate(g[key].split()):
+            for l in range(L):
+                for kv in range(2):
+                    want = bytes(row) if tok == "." else token_row(names[tok], l, kv, row)
+                    assert bytes(pvc[l, b, kv, s]) == want, (key, s)
+    assert oc.stats()["rows_copied"] == int(g["Zc.rows_copied"])
+    assert oc.refcounts().tolist() == [1, 2, 1, 3, 1, 1, 1, 1] and oc.free_list().tolist() == []
     st, Z = o.compose([c1, c2])
     assert (st, Z) == (0, 3)
     assert o.table(Z).tolist() == [int(x) for x in g["Z.table"].split()]
