@@ -297,3 +297,32 @@ def test_bench_prints_one_json_line_with_the_contract_keys():
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert set(d["cpu_baseline"]) >= {"value", "unit", "cores", "kind", "sample"} and d["cpu_baseline"]["kind"] == "oracle"
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    assert d["repeats"] >= 1 and d["timed_seconds"] > 0 and "traffic_source" in r
+    assert set(d["e2e"]) >= {"pcie_floor_ms_per_step", "frac_of_pcie_floor", "api"}
+
+
+def test_default_bench_line_carries_the_other_full_size_workloads():
+    """The headline run also measures the 70B-shaped step, the composition levels and the copy-on-write stress and
+    attaches them as roofline.per_workload (short timed regions here; the keys and the sanity of the figures)."""
+    import json
+    import os
+    import subprocess
+    import sys
+
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < (80 << 30):
+        pytest.skip("not enough free device memory for the full-size pools")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--steps", "3", "--warmup", "3",
+                          "--min-seconds", "0.05", "--no-e2e", "--no-cpu-baseline"], capture_output=True, text=True,
+                         timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
+    assert d["config"]["n_blocks"] == 32768 and d["gpu_launches"] == 3 * 12
+    pw = d["roofline"]["per_workload"]
+    assert set(pw) == {"70b", "compose_pairs", "compose_quads", "compose_all16", "compose_flat16", "cow"}
+    for name, rec in pw.items():
+        assert set(rec) >= {"achieved", "frac", "algorithmic_bytes_per_launch", "mean_launch_ms", "launches"}, name
+        assert 0.5 < rec["frac"] < 1.2 and rec["launches"] > 0, (name, rec["frac"])
+        assert abs(rec["achieved"] - rec["frac"] * d["roofline"]["peak"]) < 1e-6 * rec["achieved"]
+    assert "frac_of_measured_peak" not in pw["cow"] and pw["cow"]["counted_read_plus_written_GBps"] > pw["cow"]["achieved"]
