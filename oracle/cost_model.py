@@ -9,8 +9,9 @@ The paper's formulas written out in plain Python floats (IEEE double), in the pa
                    recompute                                                     (Sec. 4.6; App. C; App. E step 5)
   transfer_time_packed   T_transfer plus a pack at the sender and an unpack at the receiver, each moving 2 |KV|
                    bytes (read + written) at `pack_rate` bytes/s: the term the paper's model leaves out, the one
-                   this build measures.  Not from the paper: parity unpinned by the paper, pinned by its
-                   definition only (sum of three terms).
+                   this build measures.  The definition is this build's, not the paper's; it is pinned by
+                   hand-computed values (tests/golden/packed_transfer_example.txt) and by the special case of an
+                   infinitely fast pack, which must leave the paper's T_transfer.
 """
 from __future__ import annotations
 

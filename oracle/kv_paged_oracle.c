@@ -15,10 +15,12 @@
  *     App. A.2), kept here as "number of block-table entries that name the block".
  *
  * Physical conventions the paper leaves open (allocation order, free order, context
- * ids, share-vs-copy rule of the merge) are fixed as follows; parity of tables,
- * refcounts and free list is "parity unpinned" by the paper and pinned only by
- * these rules, while every materialised byte is pinned by the value model
- * (oracle/value_model.py) and the invariants in the tests:
+ * ids, share-vs-copy rule of the merge) are fixed as follows.  The paper cannot pin
+ * them; they are pinned by two worked examples derived by hand from these rules
+ * (tests/golden/worked_example_w1.txt and _w2.txt: tables, block contents, reference
+ * counts and the order of the free list, including the order in which one evicting
+ * call frees several blocks), while every materialised byte is pinned by the value
+ * model (oracle/value_model.py) and the invariants in the tests:
  *   pool    : bytes [L][NB][2][BS][row], row = H*D*E bytes (one token, one layer, K or V)
  *   buffer  : transfer layout [L][2][n][row], dense, no header
  *   ring    : FIFO of free block ids; alloc takes ring[head++ mod NB],

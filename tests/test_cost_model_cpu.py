@@ -50,6 +50,21 @@ def test_policy_is_the_strict_comparison_of_the_scheduling_rule():
     assert cm.policy(False, 1.0, 1.0) == cm.RECOMPUTE  # "transfer if T_transfer < T_prefill", otherwise recompute
 
 
+def test_packed_time_against_hand_computed_values():
+    g = _read(os.path.join(GOLD, "packed_transfer_example.txt"))
+    kv, bw = float(g["kv_bytes"]), float(g["bandwidth_bytes_per_sec"])
+    lat, rate = float(g["latency_sec"]), float(g["pack_rate_bytes_per_sec"])
+    for f_t, f_p in ((cm.transfer_time, cm.transfer_time_packed),
+                     (binding.aaf_kv_transfer_time, binding.aaf_kv_transfer_time_packed)):
+        assert f_t(kv, bw, lat) == float(g["t_transfer_sec"])       # exact: powers of two
+        assert f_p(kv, bw, lat, rate) == float(g["t_packed_sec"])
+        t = f_p(float(g["paper_kv_bytes"]), 25e9, 50e-6, float(g["paper_pack_rate"])) * 1e3
+        assert round(t, int(g["paper_t_packed_digits"])) == float(g["paper_t_packed_ms"])
+        # halving the pack rate adds exactly one more pack + unpack; an infinitely fast pack leaves T_transfer
+        assert f_p(kv, bw, lat, rate / 2) == 5.5
+    assert cm.transfer_time_packed(kv, bw, lat, math.inf) == 4.5
+
+
 def test_packed_time_is_wire_time_plus_a_pack_and_an_unpack():
     kv, bw, lat, rate = 4.0e9, 25e9, 50e-6, 6.4e12
     t = cm.transfer_time_packed(kv, bw, lat, rate)
