@@ -407,3 +407,20 @@ def test_worked_example_w2_free_order_against_the_hand_derived_values():
     assert be.o.refcounts().tolist() == ints("budget.refcount")
     assert be.o.free_list().tolist() == ints("budget.free_list")
     assert be.o.live_ctxs() == [0] and be.o.sync_status() == 0
+
+
+def test_small_batch_with_many_entries_takes_the_grid_evict_path():
+    """Two contexts (a small batch, which would travel as kernel parameters) with 70 000 table entries between
+    them (beyond what one CTA compacts): the argument records must go through memory and the grid-wide
+    count / scan / scatter must free the same blocks in the same order as the oracle."""
+    g = Geometry(1, 1, 8, 1, 2, 70000, 8, 80000)  # one token per block, 16-byte rows
+    ops = [
+        {"op": "import", "out": "a", "n": 35000, "stream": 1},
+        {"op": "fork", "ctx": "a", "k": 1, "out": ["b"]},
+        {"op": "import", "out": "c", "n": 30000, "stream": 2},
+        {"op": "evict", "ctxs": ["c", "a"]},   # frees c's 30 000 blocks; a's stay referenced by b
+        {"op": "compose", "segs": ["b", "b"], "flags": 0, "out": "bb"},
+        {"op": "evict", "ctxs": ["bb", "b"]},  # 105 000 entries on 35 000 blocks, each named three times
+    ]
+    gpu, cpu = lockstep(g, 77, ops)
+    assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
