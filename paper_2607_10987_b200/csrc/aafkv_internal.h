@@ -107,6 +107,13 @@ constexpr int SMALL_ARGS = 16;
 struct SmallInts {        // fork: children[k]; evict: ctx[n] followed by ent_off[n + 1]
     int v[2 * SMALL_ARGS + 1];
 };
+constexpr int SMALL_RECORDS = 8;   // append entries / compose segments that travel as kernel parameters
+struct SmallAppend {
+    AppendEntry e[SMALL_RECORDS];
+};
+struct SmallCompose {
+    ComposeSeg s[SMALL_RECORDS];
+};
 
 // ---- launchers (each returns cudaGetLastError() of its launches)
 // `clock` is the logical clock of the call (count of successful state-touching calls); planners stamp
@@ -118,10 +125,13 @@ cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long l
 // children_dev == nullptr: the k <= SMALL_ARGS children are in `small`
 cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
                         const SmallInts &small, long long clock, cudaStream_t st);
-cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
-                               int total_slots, int max_batch, int dry_run, long long clock, cudaStream_t st);
-cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
-                                int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st);
+// entries_dev / segs_dev == nullptr: the n (m) <= SMALL_RECORDS records are in `small`
+cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev,
+                               const SmallAppend &small, int n, int total_slots, int max_batch, int dry_run,
+                               long long clock, cudaStream_t st);
+cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, const SmallCompose &small,
+                                int m, int total_work, int total_fresh, int total_slots, int out_ctx, long long clock,
+                                cudaStream_t st);
 // args_dev == nullptr: the n <= SMALL_ARGS contexts and their entry offsets are in `small` (total <= 32768)
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,
                          int total, long long clock, int *n_launches, cudaStream_t st);

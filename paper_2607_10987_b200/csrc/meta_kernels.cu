@@ -232,11 +232,18 @@ __global__ void __launch_bounds__(256) fork_kernel(Geom g, DevState s, int paren
 //
 // scratch layout (ints): tailb[n] | need[n] | alloc_off[n]
 __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevState s,
-                                                                   const AppendEntry *__restrict__ ent_host, int n,
-                                                                   int total_slots, int max_batch, int dry_run,
-                                                                   long long clock) {
+                                                                   const AppendEntry *__restrict__ ent_host,
+                                                                   SmallAppend small, int n, int total_slots,
+                                                                   int max_batch, int dry_run, long long clock) {
     __shared__ AppendEntry sh_ent[768];
-    const AppendEntry *ent = stage_args(ent_host, n, sh_ent, 768);
+    const AppendEntry *ent;
+    if (ent_host) {
+        ent = stage_args(ent_host, n, sh_ent, 768);
+    } else {  // a small batch arrives as kernel parameters
+        if (threadIdx.x < n) sh_ent[threadIdx.x] = small.e[threadIdx.x];
+        __syncthreads();
+        ent = sh_ent;
+    }
     int *tailb = s.scratch;
     int *need = s.scratch + max_batch;
     int *alloc_off = s.scratch + 2 * max_batch;
@@ -370,11 +377,19 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 //   copy segment  : item w -> destination block nblk(off)-(off%BS>0) + w, which receives tokens
 //                   from at most two source blocks (one two-part piece per item)
 __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
-                                                                    const ComposeSeg *__restrict__ segs_host, int m,
-                                                                    int total_work, int total_fresh, int total_slots,
-                                                                    int out_ctx, long long clock) {
+                                                                    const ComposeSeg *__restrict__ segs_host,
+                                                                    SmallCompose small, int m, int total_work,
+                                                                    int total_fresh, int total_slots, int out_ctx,
+                                                                    long long clock) {
     __shared__ ComposeSeg sh_segs[512];
-    const ComposeSeg *segs = stage_args(segs_host, m, sh_segs, 512);
+    const ComposeSeg *segs;
+    if (segs_host) {
+        segs = stage_args(segs_host, m, sh_segs, 512);
+    } else {  // a few segments arrive as kernel parameters
+        if (threadIdx.x < m) sh_segs[threadIdx.x] = small.s[threadIdx.x];
+        __syncthreads();
+        segs = sh_segs;
+    }
     const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
     const bool ok = (tail - head0) >= (unsigned long long)total_fresh;
     int *out = s.tables + (long long)out_ctx * g.max_blk;
@@ -810,15 +825,18 @@ cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long 
     fork_kernel<<<grid_for(nblk * k, 256, 148), 256, 0, st>>>(g, s, parent, T, k, children_dev, small, clock);
     return cudaGetLastError();
 }
-cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev, int n,
-                               int total_slots, int max_batch, int dry_run, long long clock, cudaStream_t st) {
-    plan_append_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, entries_dev, n, total_slots, max_batch, dry_run, clock);
+cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev,
+                               const SmallAppend &small, int n, int total_slots, int max_batch, int dry_run,
+                               long long clock, cudaStream_t st) {
+    plan_append_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, entries_dev, small, n, total_slots, max_batch, dry_run,
+                                                   clock);
     return cudaGetLastError();
 }
-cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, int m, int total_work,
-                                int total_fresh, int total_slots, int out_ctx, long long clock, cudaStream_t st) {
-    plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, m, total_work, total_fresh, total_slots, out_ctx,
-                                                    clock);
+cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, const SmallCompose &small,
+                                int m, int total_work, int total_fresh, int total_slots, int out_ctx, long long clock,
+                                cudaStream_t st) {
+    plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, small, m, total_work, total_fresh, total_slots,
+                                                    out_ctx, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,

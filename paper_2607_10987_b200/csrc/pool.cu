@@ -764,7 +764,11 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     p->last_stream = st;
 
-    AppendEntry *ent = reinterpret_cast<AppendEntry *>(acquire_args(p));
+    // a small batch travels as kernel parameters, a large one through the pinned argument ring
+    SmallAppend small{};
+    const bool by_value = n <= SMALL_RECORDS;
+    AppendEntry *ent = by_value ? small.e : reinterpret_cast<AppendEntry *>(acquire_args(p));
+    const AppendEntry *ent_dev = by_value ? nullptr : ent;
     int off = 0;
     for (int i = 0; i < n; ++i) {
         const long long T = p->len[ctxs[i]];
@@ -783,8 +787,8 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             // the worst case does not fit: ask the planner (dry run) how many blocks the batch really
             // needs; only tail blocks that are still shared are copied
             unsigned long long need = 0;
-            if (launch_plan_append(p->g, p->s, ent, n, (int)slots, p->lay.max_batch, 1, p->clock, p->meta_stream) !=
-                    cudaSuccess ||
+            if (launch_plan_append(p->g, p->s, ent_dev, small, n, (int)slots, p->lay.max_batch, 1, p->clock,
+                                   p->meta_stream) != cudaSuccess ||
                 cudaStreamSynchronize(p->meta_stream) != cudaSuccess ||
                 cudaMemcpy(&need, &p->s.ctl->probe_need, sizeof(need), cudaMemcpyDeviceToHost) != cudaSuccess)
                 rc = AAF_ERR_CUDA;
@@ -794,14 +798,14 @@ int aaf_kv_append(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int32_
             charge = (long long)need;
         }
         if (rc != AAF_OK) {
-            release_args(p, p->meta_stream);
+            if (!by_value) release_args(p, p->meta_stream);
             return rc;
         }
     }
     const PlanSlot ps = begin_plan(p);
-    const cudaError_t e = launch_plan_append(p->g, ps.view, ent, n, (int)slots, p->lay.max_batch, 0, p->clock + 1,
-                                             p->meta_stream);
-    release_args(p, p->meta_stream);
+    const cudaError_t e = launch_plan_append(p->g, ps.view, ent_dev, small, n, (int)slots, p->lay.max_batch, 0,
+                                             p->clock + 1, p->meta_stream);
+    if (!by_value) release_args(p, p->meta_stream);
     if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
@@ -899,12 +903,15 @@ int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t fl
     const int rc0 = ensure_free(p, fresh, st);
     if (rc0 != AAF_OK) return rc0;
     p->last_stream = st;
-    ComposeSeg *dev_rec = reinterpret_cast<ComposeSeg *>(acquire_args(p));
-    memcpy(dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
+    // a few segments travel as kernel parameters, more through the pinned argument ring
+    SmallCompose small{};
+    const bool by_value = m <= SMALL_RECORDS;
+    ComposeSeg *dev_rec = by_value ? nullptr : reinterpret_cast<ComposeSeg *>(acquire_args(p));
+    memcpy(by_value ? small.s : dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
     const PlanSlot ps = begin_plan(p);
-    const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, m, (int)work, (int)fresh, (int)slots, c,
+    const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, small, m, (int)work, (int)fresh, (int)slots, c,
                                               p->clock + 1, p->meta_stream);
-    release_args(p, p->meta_stream);
+    if (!by_value) release_args(p, p->meta_stream);
     if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
     p->clock += 1;
     p->meta_launches += 1;
