@@ -324,7 +324,8 @@ def compose_levels(args, peak, steps, warmup, copy_all=False):
     by_level = {}
     for o in (o for o in ops if o["op"] == "compose"):
         by_level.setdefault(o["level"], []).append(o)
-    acc = {k: {"ms": 0.0, "kernel_ms": 0.0, "launches": 0, "bytes": 0, "ops": 0, "b2b_ms": 0.0, "b2b_bytes": 0}
+    acc = {k: {"ms": 0.0, "kernel_ms": 0.0, "launches": 0, "bytes": 0, "ops": 0, "b2b_ms": 0.0, "b2b_bytes": 0,
+               "bat_ms": 0.0, "bat_kernel_ms": 0.0, "bat_bytes": 0, "bat_launches": 0}
            for k in by_level}
 
     def run_level(level, made):
@@ -334,11 +335,24 @@ def compose_levels(args, peak, steps, warmup, copy_all=False):
             names[o["out"]] = c
             made.append(c)
 
-    for it in range(warmup + 2 * steps):
+    def run_level_batched(level, made):  # the whole level as ONE call: one planner launch, one copy launch
+        st, outs = be.o.compose_batch([[names[x] for x in o["segs"]] for o in by_level[level]],
+                                      by_level[level][0]["flags"])
+        assert st == 0
+        for o, c in zip(by_level[level], outs):
+            names[o["out"]] = c
+        made += outs
+
+    for it in range(warmup + 3 * steps):
         made = []
-        kernel_pass = it < warmup + steps  # first the per-kernel events, then the back-to-back levels
+        kernel_pass = it < warmup + steps  # first the per-kernel events, then the back-to-back levels, then batches
+        batched_pass = it >= warmup + 2 * steps
         for level in by_level:
-            if kernel_pass:
+            if batched_pass:
+                ms, dms, dl, b = timed_ops(be.o, lambda: run_level_batched(level, made))
+                a = acc[level]
+                a["bat_ms"] += ms; a["bat_kernel_ms"] += dms["compose"]; a["bat_bytes"] += b; a["bat_launches"] += dl["compose"]
+            elif kernel_pass:
                 ms, dms, dl, b = timed_ops(be.o, lambda: run_level(level, made))
                 if it >= warmup:
                     a = acc[level]
@@ -362,7 +376,12 @@ def compose_levels(args, peak, steps, warmup, copy_all=False):
         lvl = 2 * a["b2b_bytes"] / (a["b2b_ms"] * 1e-3) / 1e9
         rec.update({"composes_per_level": len(by_level[level]), "copied_GB_per_compose": a["bytes"] / a["ops"] / 1e9,
                     "level_GBps": lvl, "level_frac": lvl / peak, "level_ms": a["b2b_ms"] / steps,
-                    "level_note": "the level's composes issued back to back, events around the level"})
+                    "level_note": "the level's composes issued back to back, events around the level",
+                    "batched_level_GBps": 2 * a["bat_bytes"] / (a["bat_ms"] * 1e-3) / 1e9,
+                    "batched_kernel_GBps": 2 * a["bat_bytes"] / (a["bat_kernel_ms"] * 1e-3) / 1e9,
+                    "batched_kernel_frac": 2 * a["bat_bytes"] / (a["bat_kernel_ms"] * 1e-3) / 1e9 / peak,
+                    "batched_launches_per_level": a["bat_launches"] / steps,
+                    "batched_note": "the whole level as one aaf_kv_compose_batch call: one copy launch"})
         out[level] = rec
     del be
     torch.cuda.empty_cache()

@@ -198,6 +198,18 @@ int aaf_kv_append(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, const int
 int aaf_kv_compose(aaf_kv_pool *pool, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
                    void *stream);
 
+/* compose, batched -- n_out independent merges (Alg. "Restricted-KV-Merge", concatenation branch) in one call:
+ * merge i concatenates segs[seg_off[i] .. seg_off[i + 1]) (seg_off has n_out + 1 entries, seg_off[0] = 0, every
+ * merge at least one segment).  When it succeeds the result is exactly that of the for-loop of aaf_kv_compose
+ * over i -- the same handles (the n_out smallest free ones, in order), the same block tables (each merge takes its
+ * fresh blocks behind those of the merges before it), the same catalog stamps -- but with one planner launch and
+ * ONE copy launch for all merges, so that a level of small merges (the agents of a workflow merged in pairs)
+ * does not pay the launch ramp per merge.  Segments must be live before the call (a result of the same batch
+ * cannot be a segment).  The batch is all-or-nothing: any error leaves every merge undone.  seg_off, segs host;
+ * out_ctxs (host, n_out entries).  Errors: as aaf_kv_compose; OOM_CTX / OOM_BLOCKS / TOO_MANY count the whole batch. */
+int aaf_kv_compose_batch(aaf_kv_pool *pool, int32_t n_out, const int32_t *seg_off, const aaf_ctx_t *segs,
+                         uint32_t flags, aaf_ctx_t *out_ctxs, void *stream);
+
 /* evict -- Alg. "KV-Evict", release step: every block-table entry of every listed context drops
  * one reference; blocks that reach 0 return to the ring's tail in (context, table position)
  * order; the handles become free.  Victim selection is the caller's policy.  ctxs is a host

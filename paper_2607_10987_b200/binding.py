@@ -76,6 +76,7 @@ SYMBOLS = {
     "aaf_kv_fork": (C.c_int, [_vp, _i32, _i32, _p32, _vp]),
     "aaf_kv_append": (C.c_int, [_vp, _i32, _p32, _p32, C.POINTER(_vp), _vp]),
     "aaf_kv_compose": (C.c_int, [_vp, _i32, _p32, _u32, _p32, _vp]),
+    "aaf_kv_compose_batch": (C.c_int, [_vp, _i32, _p32, _p32, _u32, _p32, _vp]),
     "aaf_kv_evict": (C.c_int, [_vp, _i32, _p32, _vp]),
     "aaf_kv_materialize_host": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import_host": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _vp, _sz, _p32, _vp]),
@@ -139,6 +140,8 @@ def aaf_kv_import(pool, src, desc, out_ctx, stream): return _fn("aaf_kv_import")
 def aaf_kv_fork(pool, parent, k, out_children, stream): return _fn("aaf_kv_fork")(pool, parent, k, out_children, stream)
 def aaf_kv_append(pool, n, ctxs, n_new, srcs, stream): return _fn("aaf_kv_append")(pool, n, ctxs, n_new, srcs, stream)
 def aaf_kv_compose(pool, m, segs, flags, out_ctx, stream): return _fn("aaf_kv_compose")(pool, m, segs, flags, out_ctx, stream)
+def aaf_kv_compose_batch(pool, n_out, seg_off, segs, flags, out_ctxs, stream):
+    return _fn("aaf_kv_compose_batch")(pool, n_out, seg_off, segs, flags, out_ctxs, stream)
 def aaf_kv_evict(pool, n, ctxs, stream): return _fn("aaf_kv_evict")(pool, n, ctxs, stream)
 def aaf_kv_materialize_host(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream):
     return _fn("aaf_kv_materialize_host")(pool, ctx, t0, t1, dst_host, dst_bytes, staging, staging_bytes, out_desc, stream)
@@ -301,6 +304,19 @@ class KVPool:
         out = C.c_int32(-1)
         st = aaf_kv_compose(self.h, m, a, flags, C.byref(out), self._stream())
         return st, (out.value if st == AAF_OK else None)
+
+    def compose_batch(self, seg_lists, flags=0):
+        """seg_lists: one list of segment handles per merge; returns (status, [result handles])."""
+        n_out = len(seg_lists)
+        offs, flat = [0], []
+        for segs in seg_lists:
+            flat += list(segs)
+            offs.append(len(flat))
+        a = (C.c_int32 * (n_out + 1))(*offs)
+        b = (C.c_int32 * max(len(flat), 1))(*flat)
+        out = (C.c_int32 * max(n_out, 1))()
+        st = aaf_kv_compose_batch(self.h, n_out, a, b, flags, out, self._stream())
+        return st, (list(out[:n_out]) if st == AAF_OK else None)
 
     def evict(self, ctxs):
         n = len(ctxs)

@@ -85,18 +85,21 @@ struct AppendEntry {      // 32 bytes
     int piece_off;        // first piece slot of this entry (slot 0 = COW piece)
     int pad;
 };
-struct ComposeSeg {       // 48 bytes
+struct ComposeSeg {       // 56 bytes; one per segment of every merge of a batch
     long long T;          // tokens of the segment
-    long long off;        // token offset of the segment in the result
+    long long off;        // token offset of the segment in its result
     int ctx;
     int mode;             // 0 = share (aligned), 1 = copy
-    int share_tail;       // share mode: 1 = partial tail shared by reference (last segment)
-    int work_off;         // first flattened work item of the segment
-    int fresh_start;      // rank (from ring head) of the first fresh block the segment allocates
-    int piece_off;        // first piece slot of the segment
+    int share_tail;       // share mode: 1 = partial tail shared by reference (last segment of its result)
+    int work_off;         // first flattened work item of the segment (over the whole batch)
+    int fresh_start;      // rank (from ring head, over the whole batch) of the first fresh block the segment allocates
+    int piece_off;        // first piece slot of the segment (over the whole batch)
     int dst_tbl_start;    // share mode: first result-table index written
-    int pad;
+    int out_ctx;          // handle of the result this segment belongs to
+    int out_index;        // which result of the batch (its logical clock is the call's clock + out_index)
+    int first_ctx;        // last segment of a result only: handle of the result's first segment, else -1
 };
+static_assert(sizeof(ComposeSeg) == 56, "ComposeSeg layout");
 struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
     int n;
     int total;
@@ -129,8 +132,9 @@ cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long 
 cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEntry *entries_dev,
                                const SmallAppend &small, int n, int total_slots, int max_batch, int dry_run,
                                long long clock, cudaStream_t st);
+// `clock` is the logical clock of the batch's first merge; merge i of the batch is stamped clock + i
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, const SmallCompose &small,
-                                int m, int total_work, int total_fresh, int total_slots, int out_ctx, long long clock,
+                                int m, int total_work, int total_fresh, int total_slots, long long clock,
                                 cudaStream_t st);
 // args_dev == nullptr: the n <= SMALL_ARGS contexts and their entry offsets are in `small` (total <= 32768)
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,

@@ -369,18 +369,21 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_append_kernel(Geom g, DevSt
 }
 
 // ------------------------------------------------------------------------------------------
-// compose: flattened over the work items of all segments (host supplies the prefix sums of the
-// lengths, which it knows; block ids come from the ring at rank offsets from the old head).
+// compose: flattened over the work items of all segments of all merges of the batch (host supplies the prefix
+// sums of the lengths, which it knows; block ids come from the ring at rank offsets from the old head).
 //   share segment : item w < full -> share entry w; item w == full -> the partial tail (shared by
 //                   reference if it ends the result, else re-packed into a fresh block through the
 //                   segment's single piece slot)
 //   copy segment  : item w -> destination block nblk(off)-(off%BS>0) + w, which receives tokens
 //                   from at most two source blocks (one two-part piece per item)
+// A batch of merges is the for-loop over its merges: every merge reads only contexts that were live before the
+// call, writes only its own fresh blocks and its own table, and takes its fresh blocks behind those of the merges
+// before it; reference counts add up in any order; the catalog is stamped as the loop would stamp it (merge i at
+// clock + i, a source's last access = the latest merge that read it).
 __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevState s,
                                                                     const ComposeSeg *__restrict__ segs_host,
                                                                     SmallCompose small, int m, int total_work,
-                                                                    int total_fresh, int total_slots, int out_ctx,
-                                                                    long long clock) {
+                                                                    int total_fresh, int total_slots, long long clock) {
     __shared__ ComposeSeg sh_segs[512];
     const ComposeSeg *segs;
     if (segs_host) {
@@ -392,7 +395,6 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
     }
     const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
     const bool ok = (tail - head0) >= (unsigned long long)total_fresh;
-    int *out = s.tables + (long long)out_ctx * g.max_blk;
     if (!ok) {
         for (int sl = threadIdx.x; sl < total_slots; sl += blockDim.x) clear_piece(s.pieces[sl]);
     }
@@ -406,6 +408,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
         const ComposeSeg sg = segs[lo];
         const int w = it - sg.work_off;
         const int *st = s.tables + (long long)sg.ctx * g.max_blk;
+        int *out = s.tables + (long long)sg.out_ctx * g.max_blk;
         if (sg.mode == 0) {
             const long long full = sg.T / g.BS;
             const int rem = (int)(sg.T % g.BS);
@@ -451,16 +454,20 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_compose_kernel(Geom g, DevS
     if (ok && s.cat_len)
         for (int i = threadIdx.x; i < m; i += blockDim.x) {  // every occurrence of a segment is one read
             atomicAdd(&s.cat_reuse[segs[i].ctx], 1ull);
-            s.cat_last[segs[i].ctx] = clock;
+            atomicMax(&s.cat_last[segs[i].ctx], clock + segs[i].out_index);
         }
     __syncthreads();
+    if (ok && s.cat_len)
+        for (int i = threadIdx.x; i < m; i += blockDim.x)  // the last segment of a result registers the result
+            if (segs[i].first_ctx >= 0)
+                catalog_born(s, segs[i].out_ctx, segs[i].off + segs[i].T, clock + segs[i].out_index, 3,
+                             segs[i].first_ctx);
     if (threadIdx.x == 0) {
         if (!ok) {
             set_status(s.ctl, AAF_ERR_CORRUPT, 6);
         } else {
             s.ctl->head = head0 + total_fresh;
             note_alloc(s.ctl, g, head0 + total_fresh, tail);
-            if (s.cat_len) catalog_born(s, out_ctx, segs[m - 1].off + segs[m - 1].T, clock, 3, segs[0].ctx);
         }
     }
 }
@@ -833,10 +840,10 @@ cudaError_t launch_plan_append(const Geom &g, const DevState &s, const AppendEnt
     return cudaGetLastError();
 }
 cudaError_t launch_plan_compose(const Geom &g, const DevState &s, const ComposeSeg *segs_dev, const SmallCompose &small,
-                                int m, int total_work, int total_fresh, int total_slots, int out_ctx, long long clock,
+                                int m, int total_work, int total_fresh, int total_slots, long long clock,
                                 cudaStream_t st) {
     plan_compose_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, segs_dev, small, m, total_work, total_fresh, total_slots,
-                                                    out_ctx, clock);
+                                                    clock);
     return cudaGetLastError();
 }
 cudaError_t launch_evict(const Geom &g, const DevState &s, const EvictArgs *args_dev, const SmallInts &small, int n,

@@ -857,71 +857,106 @@ int aaf_kv_append_host(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const i
     return rc;
 }
 
-int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
-                   void *stream) {
-    AAF_RANGE("aaf_kv_compose");
-    if (!p || m < 1 || !segs || !out_ctx || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
-    if (p->broken) return AAF_ERR_CUDA;
-    if (m > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+// n_out merges in one planner launch and one copy launch: merge i concatenates segs[seg_off[i] .. seg_off[i + 1])
+static int compose_impl(aaf_kv_pool *p, int32_t n_out, const int32_t *seg_off, const aaf_ctx_t *segs, uint32_t flags,
+                        aaf_ctx_t *out_ctxs, cudaStream_t st) {
+    const int m = seg_off[n_out];
+    if (m > p->lay.max_batch || n_out > p->lay.max_batch) return AAF_ERR_TOO_MANY;
     for (int i = 0; i < m; ++i)
         if (!is_live(p, segs[i])) return AAF_ERR_BAD_CTX;
     const bool copy_all = (flags & AAF_COMPOSE_COPY_ALL) != 0;
     const int BS = p->g.BS;
     // everything but the block ids follows from the lengths
     std::vector<ComposeSeg> rec((size_t)m);
-    long long off = 0, fresh = 0, work = 0, slots = 0, tbl = 0, copied_tokens = 0;
-    for (int i = 0; i < m; ++i) {
-        const long long T = p->len[segs[i]];
-        ComposeSeg &r = rec[(size_t)i];
-        memset(&r, 0, sizeof(r));
-        r.T = T; r.off = off; r.ctx = segs[i];
-        r.work_off = (int)work; r.fresh_start = (int)fresh; r.piece_off = (int)slots;
-        if (!copy_all && off % BS == 0) {
-            r.mode = 0;
-            r.share_tail = (i == m - 1);
-            r.dst_tbl_start = (int)tbl;
-            const long long items = nblk_of(p, T);
-            work += items;
-            if (T % BS && i != m - 1) { fresh += 1; slots += 1; copied_tokens += T % BS; }
-        } else {
-            r.mode = 1;
-            const long long items = (off + T - 1) / BS - off / BS + 1;
-            work += items;
-            slots += items;  // one two-part piece per destination block
-            copied_tokens += T;
-            fresh += nblk_of(p, off + T) - nblk_of(p, off);
+    std::vector<long long> out_len((size_t)n_out);
+    long long fresh = 0, work = 0, slots = 0, copied_tokens = 0;
+    for (int o = 0; o < n_out; ++o) {
+        long long off = 0, tbl = 0;
+        const int s0 = seg_off[o], s1 = seg_off[o + 1];
+        for (int i = s0; i < s1; ++i) {
+            const long long T = p->len[segs[i]];
+            const bool last = i == s1 - 1;
+            ComposeSeg &r = rec[(size_t)i];
+            memset(&r, 0, sizeof(r));
+            r.T = T; r.off = off; r.ctx = segs[i];
+            r.work_off = (int)work; r.fresh_start = (int)fresh; r.piece_off = (int)slots;
+            r.out_index = o;
+            r.first_ctx = last ? segs[s0] : -1;
+            if (!copy_all && off % BS == 0) {
+                r.mode = 0;
+                r.share_tail = last;
+                r.dst_tbl_start = (int)tbl;
+                work += nblk_of(p, T);
+                if (T % BS && !last) { fresh += 1; slots += 1; copied_tokens += T % BS; }
+            } else {
+                r.mode = 1;
+                const long long items = (off + T - 1) / BS - off / BS + 1;
+                work += items;
+                slots += items;  // one two-part piece per destination block
+                copied_tokens += T;
+                fresh += nblk_of(p, off + T) - nblk_of(p, off);
+            }
+            off += T;
+            tbl = nblk_of(p, off);
         }
-        off += T;
-        tbl = nblk_of(p, off);
+        if (nblk_of(p, off) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+        out_len[(size_t)o] = off;
     }
-    if (nblk_of(p, off) > p->g.max_blk) return AAF_ERR_TOO_LONG;
-    if (slots > p->lay.max_pieces) return AAF_ERR_TOO_MANY;
-    const int c = smallest_free_ctx(p);
-    if (c < 0) return AAF_ERR_OOM_CTX;
-    DeviceGuard guard(p->device);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (slots > p->lay.max_pieces || work >= (1ll << 31)) return AAF_ERR_TOO_MANY;
+    if (p->g.max_ctx - p->live_ctx < n_out) return AAF_ERR_OOM_CTX;
     const int rc0 = ensure_free(p, fresh, st);
     if (rc0 != AAF_OK) return rc0;
     p->last_stream = st;
+    std::vector<int> handles((size_t)n_out);
+    int c = -1;
+    for (int o = 0; o < n_out; ++o) {  // the n_out smallest free handles, in order: what the loop of merges would take
+        c = smallest_free_ctx(p, c + 1);
+        handles[(size_t)o] = c;
+    }
+    for (int i = 0; i < m; ++i) rec[(size_t)i].out_ctx = handles[(size_t)rec[(size_t)i].out_index];
     // a few segments travel as kernel parameters, more through the pinned argument ring
     SmallCompose small{};
     const bool by_value = m <= SMALL_RECORDS;
     ComposeSeg *dev_rec = by_value ? nullptr : reinterpret_cast<ComposeSeg *>(acquire_args(p));
     memcpy(by_value ? small.s : dev_rec, rec.data(), sizeof(ComposeSeg) * (size_t)m);
     const PlanSlot ps = begin_plan(p);
-    const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, small, m, (int)work, (int)fresh, (int)slots, c,
+    const cudaError_t e = launch_plan_compose(p->g, ps.view, dev_rec, small, m, (int)work, (int)fresh, (int)slots,
                                               p->clock + 1, p->meta_stream);
     if (!by_value) release_args(p, p->meta_stream);
     if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
-    p->clock += 1;
+    p->clock += n_out;  // merge i of the batch is the call with clock + 1 + i
     p->meta_launches += 1;
     p->free_lb -= fresh;
-    p->len[c] = off;
-    p->live_ctx += 1;
-    *out_ctx = c;
+    for (int o = 0; o < n_out; ++o) {
+        p->len[handles[(size_t)o]] = out_len[(size_t)o];
+        out_ctxs[o] = handles[(size_t)o];
+    }
+    p->live_ctx += n_out;
     const int rc_copy = run_copy(p, ps, AAF_OP_COMPOSE, (int)slots, copied_tokens, st);
     end_copy(p, ps, st);
     return rc_copy;
+}
+
+int aaf_kv_compose(aaf_kv_pool *p, int32_t m, const aaf_ctx_t *segs, uint32_t flags, aaf_ctx_t *out_ctx,
+                   void *stream) {
+    AAF_RANGE("aaf_kv_compose");
+    if (!p || m < 1 || !segs || !out_ctx || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
+    DeviceGuard guard(p->device);
+    const int32_t seg_off[2] = {0, m};
+    return compose_impl(p, 1, seg_off, segs, flags, out_ctx, static_cast<cudaStream_t>(stream));
+}
+
+int aaf_kv_compose_batch(aaf_kv_pool *p, int32_t n_out, const int32_t *seg_off, const aaf_ctx_t *segs, uint32_t flags,
+                         aaf_ctx_t *out_ctxs, void *stream) {
+    AAF_RANGE("aaf_kv_compose_batch");
+    if (!p || n_out < 1 || !seg_off || !segs || !out_ctxs || (flags & ~AAF_COMPOSE_COPY_ALL)) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
+    if (seg_off[0] != 0) return AAF_ERR_INVALID_ARG;
+    for (int o = 0; o < n_out; ++o)
+        if (seg_off[o + 1] <= seg_off[o]) return AAF_ERR_INVALID_ARG;  // every merge has at least one segment
+    DeviceGuard guard(p->device);
+    return compose_impl(p, n_out, seg_off, segs, flags, out_ctxs, static_cast<cudaStream_t>(stream));
 }
 
 int aaf_kv_evict(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, void *stream) {

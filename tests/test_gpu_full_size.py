@@ -138,6 +138,43 @@ def test_config3_compose_levels_value_model_all_layers(copy_all):
     assert sh.vm.ctx[max(sh.vm.ctx)] == sh.vm.ctx[max(sh.vm.ctx) - 1] and len(sh.vm.ctx[max(sh.vm.ctx)]) == sum(lens)
 
 
+@pytest.mark.parametrize("copy_all", [False, True])
+def test_config3_levels_as_batches_8b(copy_all):
+    """The composition workload with every level issued as ONE batched call (8 pairs, 4 quads): tables, reference
+    counts, free list, catalog and the bytes of the sampled layer equal the oracle's loop of single merges."""
+    from tests.helpers import OracleBackend
+
+    g, seed, ops, lens = configs.config3(configs.LLAMA8B, copy_all=copy_all)
+    if not _fits(g, 16):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    layers = [11]
+    order = configs.free_order(seed, g.n_blocks)
+    gpu = GpuBackend(g, seed, free_order=order, init_fill="zero")
+    cpu = OracleBackend(g, seed, layers=layers, free_order=order, init_fill="zero")
+    names = {}
+    for o in (o for o in ops if o["op"] == "import"):
+        for be in (gpu, cpu):
+            st, c = be.imp(be.payload(seed, o["stream"], o["n"]), o["n"])
+            assert st == 0
+        names[o["out"]] = c
+    for level in ("pairs", "quads", "all16", "flat16"):
+        batch = [o for o in ops if o["op"] == "compose" and o["level"] == level]
+        st, outs = gpu.o.compose_batch([[names[x] for x in o["segs"]] for o in batch], batch[0]["flags"])
+        assert st == 0
+        for o, c in zip(batch, outs):
+            assert cpu.compose([names[x] for x in o["segs"]], o["flags"]) == (0, c)
+            names[o["out"]] = c
+        assert gpu.snapshot() == cpu.snapshot(), level
+        assert gpu.o.catalog() == cpu.o.catalog(), level
+    assert gpu.o.stats()["copy_launches"]["compose"] == 4
+    assert np.array_equal(gpu.pool_layers(layers), cpu.o.pool_view())
+    n = sum(lens)
+    for name in ("all_tree", "all_flat"):
+        got = gpu.buf_layers(gpu.materialize(names[name], 0, n)[1], n, layers).reshape(-1)
+        assert np.array_equal(got, cpu.materialize(names[name], 0, n)[1])
+    assert gpu.o.sync_status() == 0
+
+
 def test_config2_host_buffer_path_value_model_all_layers():
     """The end-to-end form of the 8B step, as the benchmark times it: every input arrives from pinned host memory
     through the library's host-buffer calls (chunked import, chunked materialize, append from host buffers), on

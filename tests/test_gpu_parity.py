@@ -424,3 +424,74 @@ def test_small_batch_with_many_entries_takes_the_grid_evict_path():
     ]
     gpu, cpu = lockstep(g, 77, ops)
     assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# aaf_kv_compose_batch: several merges in one planner launch and one copy launch == the loop of single merges
+
+
+def _merge_pool(seed, lens, g=None):
+    g = g or Geometry(3, 4, 64, 16, 2, 512, 40, 96)  # 512-byte rows, 8 KiB runs
+    order = configs.free_order(seed, g.n_blocks)
+    gpu = GpuBackend(g, seed, free_order=order)
+    cpu = OracleBackend(g, seed, free_order=order)
+    for i, n in enumerate(lens):
+        for be in (gpu, cpu):
+            assert be.imp(be.payload(seed, 1 + i, n), n) == (0, i)
+    return g, gpu, cpu
+
+
+@pytest.mark.parametrize("flags", [0, configs.COMPOSE_COPY_ALL])
+def test_compose_batch_equals_the_loop_of_single_merges(flags):
+    lens = [37, 64, 16, 5, 100, 48, 33, 1, 80, 250]
+    g, gpu, cpu = _merge_pool(31, lens)
+    # a source used by several merges, an aligned first segment, a merge of one (== fork), a long merge, repeats
+    batch = [[0, 1], [1, 2, 3], [4], [2, 2, 5, 0], [9, 8, 7, 6, 5, 4, 3], [1, 0]]
+    st, outs = gpu.o.compose_batch(batch, flags)
+    assert st == 0
+    want = []
+    for segs in batch:
+        st_c, c = cpu.compose(segs, flags)
+        assert st_c == 0
+        want.append(c)
+    assert outs == want
+    assert gpu.snapshot() == cpu.snapshot()
+    assert gpu.o.catalog() == cpu.o.catalog()
+    same_catalog_export(gpu, cpu)
+    assert np.array_equal(gpu.pool_layers(range(g.n_layers)), cpu.o.pool_view())
+    for c in outs:
+        n = cpu.o.ctx_len(c)
+        assert np.array_equal(gpu.buf_layers(gpu.materialize(c, 0, n)[1], n, range(g.n_layers)).reshape(-1),
+                              cpu.materialize(c, 0, n)[1])
+    gs, cs = gpu.o.stats(), cpu.o.stats()
+    assert gs["copy_launches"]["compose"] == 1 and gs["payload_bytes"] == cs["rows_copied"] * g.row
+    # results of a batch are ordinary contexts: merge them again, as one more batch, then evict everything
+    st, outs2 = gpu.o.compose_batch([outs[:3], outs[3:]], flags)
+    assert st == 0
+    assert [cpu.compose(outs[:3], flags)[1], cpu.compose(outs[3:], flags)[1]] == outs2
+    everything = cpu.o.live_ctxs()
+    assert gpu.evict(everything)[0] == 0 and cpu.evict(everything)[0] == 0
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+    assert sorted(gpu.o.free_list().tolist()) == list(range(g.n_blocks))
+
+
+def test_compose_batch_is_all_or_nothing():
+    from paper_2607_10987_b200 import binding
+
+    lens = [700, 700, 90, 21]
+    g, gpu, cpu = _merge_pool(32, lens, Geometry(2, 4, 64, 16, 2, 160, 6, 90))  # 90-block tables, 160 blocks, 6 handles
+    before = gpu.snapshot()
+    assert before == cpu.snapshot()
+    # second merge too long (1400 tokens = 88 blocks fits, 1490 = 94 does not); first merge alone would succeed
+    assert gpu.o.compose_batch([[2, 3], [0, 1, 2]], 0)[0] == binding.AAF_ERR_TOO_LONG
+    # not enough blocks for both copies: 96 blocks are live, 64 free; each copy-all merge of [0, 3] needs 46
+    assert gpu.o.compose_batch([[0, 3], [0, 3]], configs.COMPOSE_COPY_ALL)[0] == binding.AAF_ERR_OOM_BLOCKS
+    # three results but only two free handles
+    assert gpu.o.compose_batch([[2], [3], [2, 3]], 0)[0] == binding.AAF_ERR_OOM_CTX
+    assert gpu.o.compose_batch([[2, 3], [5]], 0)[0] == binding.AAF_ERR_BAD_CTX
+    assert gpu.o.compose_batch([[2, 3], []], 0)[0] == binding.AAF_ERR_INVALID_ARG
+    assert gpu.snapshot() == before and gpu.o.catalog() == cpu.o.catalog()
+    # and one of them alone goes through, identically on both sides
+    assert gpu.o.compose_batch([[0, 3]], configs.COMPOSE_COPY_ALL) == (0, [4])
+    assert cpu.compose([0, 3], configs.COMPOSE_COPY_ALL) == (0, 4)
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
