@@ -270,7 +270,7 @@ int run_copy(aaf_kv_pool *p, const PlanSlot &ps, int cls, int n_slots, long long
     const long long avg_piece = n_slots > 0 ? payload_tokens * p->g.row / n_slots : 0;
     if (n_slots <= 0) return AAF_OK;
     if (p->last_copy_event && st != p->last_copy_stream) {  // a different stream: serialise behind the last copy launch
-        if (cudaStreamWaitEvent(st, p->last_copy_event, 0) != cudaSuccess) return AAF_ERR_CUDA;
+        if (cudaStreamWaitEvent(st, p->last_copy_event, 0) != cudaSuccess) return broke(p);
         p->last_copy_stream = st;  // the wait is queued; later launches of this operator need not repeat it
     }
     TimedLaunch t{};
