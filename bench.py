@@ -260,13 +260,14 @@ def timed_ops(pool, fn, meta=False):
     return e0.elapsed_time(e1), dms, dl, s1["payload_bytes"] - s0["payload_bytes"]
 
 
-def cow_stress(args, peak, steps, warmup):
+def cow_stress(args, peak, steps, warmup, n_layers=32):
     """Copy-on-write stress: one unaligned 8187-token context forked to 1024 children, one batched 1-token append,
     so 1024 children each copy the 11 valid rows of the shared partial tail block.  All children read the same
-    11 source rows (they stay in the L2), so the DRAM side of this kernel is its writes."""
+    11 source rows (they stay in the L2), so the DRAM side of this kernel is its writes.  n_layers = 32: the
+    8B-shaped rows; 80: the 70B-shaped ones."""
     from tests.gpu_backend import GpuBackend
 
-    g = configs.Geometry(32, 8, 128, 16, 2, 4096, 1100, 1024)
+    g = configs.Geometry(n_layers, 8, 128, 16, 2, 2048 if n_layers > 32 else 4096, 1100, 1024)
     seed = configs.SEED_BASE + 6
     be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False,
                     max_batch=1024)
@@ -296,7 +297,7 @@ def cow_stress(args, peak, steps, warmup):
                 "frac_of_nominal_8TBps": written / 8000.0, "traffic": rec["algorithmic_bytes_per_launch"] / 2,
                 "traffic_source": "modelled: the bytes written (the 11 shared source rows are read from the L2)",
                 "note": "achieved = bytes written per second (DRAM side); the 1024 children read the same 11 rows",
-                "children": kids_n, "rows_copied_per_child": T % g.block_size,
+                "children": kids_n, "rows_copied_per_child": T % g.block_size, "n_layers": n_layers,
                 "fork_1024_ms": acc["fork_ms"] / steps, "evict_1024_plus_1_ctx_ms": acc["evict_ms"] / steps})
     del be
     return rec
@@ -408,6 +409,7 @@ def extra_report(args):
 
     if args.workload == "cow":
         out.update(cow_stress(args, peak, args.steps, args.warmup))
+        out["llama70b_rows"] = cow_stress(args, peak, args.steps, args.warmup, n_layers=80)
     elif args.workload == "compose":
         out["share"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=False)
         out["copy_all"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=True)
@@ -834,6 +836,7 @@ def main():
         for name, lv in compose_levels(args, peak, k, 2, copy_all=False).items():
             pw["compose_" + name] = lv
         pw["cow"] = cow_stress(args, peak, k, 2)
+        pw["cow_70b"] = cow_stress(args, peak, k, 2, n_layers=80)
         roofline["per_workload"] = pw
 
     if rank != 0:
