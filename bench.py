@@ -303,6 +303,57 @@ def cow_stress(args, peak, steps, warmup, n_layers=32):
     return rec
 
 
+def suffix_transfers(args, peak, steps, warmup):
+    """Partial transfers (Sec. 5.4: only the subset of a state that a consumer needs is sent): 16 agents share an
+    8187-token prefix that the receiver already holds, so only each agent's 512-token continuation is packed, and
+    unpacked at the other end.  Sixteen 64 MiB transfers, issued one call each and as ONE batched call."""
+    import torch
+
+    from tests.gpu_backend import GpuBackend
+
+    g = configs.Geometry(32, 8, 128, 16, 2, 8192, 64, 1024)
+    seed, T, agents, n_new = configs.SEED_BASE + 2, 8187, 16, 512
+    be = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), engine=args.engine, init_fill=False)
+    pool = be.o
+    st, root = be.imp(be.payload(seed, 1, T), T)
+    st, kids = be.fork(root, agents)
+    assert be.append(kids, [n_new] * agents, [be.payload(seed, 2 + i, n_new) for i in range(agents)])[0] == 0
+    bufs = [torch.empty(n_new * g.bpt, dtype=torch.uint8, device=pool.device) for _ in range(agents)]
+    acc = {k: {"ms": 0.0, "kernel_ms": 0.0, "bytes": 0, "launches": 0} for k in
+           ("pack_loop", "pack_batch", "unpack_loop", "unpack_batch")}
+
+    def note(key, r):
+        ms, dms, dl, b = r
+        a = acc[key]
+        a["ms"] += ms; a["kernel_ms"] += sum(dms.values()); a["bytes"] += b; a["launches"] += sum(dl.values())
+
+    for it in range(warmup + steps):
+        res = {}
+        r1 = timed_ops(pool, lambda: [pool.materialize(k, T, T + n_new, out=b) for k, b in zip(kids, bufs)])
+        r2 = timed_ops(pool, lambda: res.update(m=pool.materialize_batch(kids, [T] * agents, [T + n_new] * agents, bufs)))
+        assert res["m"] == 0
+        got = []
+        r3 = timed_ops(pool, lambda: got.extend(pool.imp(b, n_new)[1] for b in bufs))
+        pool.evict(got)
+        r4 = timed_ops(pool, lambda: res.update(i=pool.import_batch(bufs, [n_new] * agents)))
+        assert res["i"][0] == 0
+        pool.evict(res["i"][1])
+        if it >= warmup:
+            for key, r in (("pack_loop", r1), ("pack_batch", r2), ("unpack_loop", r3), ("unpack_batch", r4)):
+                note(key, r)
+    assert pool.sync_status() == 0
+    out = {"transfers": agents, "tokens_each": n_new, "bytes_each_MiB": n_new * g.bpt / 2**20}
+    for key, a in acc.items():
+        rec = kernel_record(2 * a["bytes"], a["kernel_ms"], a["launches"], peak)
+        rec.update({"launches_per_pass": a["launches"] / steps,
+                    "whole_pass_GBps": 2 * a["bytes"] / (a["ms"] * 1e-3) / 1e9,
+                    "whole_pass_note": "events around the 16 calls (or the one batched call), host latency included"})
+        out[key] = rec
+    del be
+    torch.cuda.empty_cache()
+    return out
+
+
 def compose_levels(args, peak, steps, warmup, copy_all=False):
     """Composition workload: 16 contexts of 1024..4096 tokens (none block-aligned) composed in pairs, quads, all 16
     (tree) and flat.  Per level: the copy kernel's rate from the library's events, and the level's throughput with
@@ -410,6 +461,8 @@ def extra_report(args):
     if args.workload == "cow":
         out.update(cow_stress(args, peak, args.steps, args.warmup))
         out["llama70b_rows"] = cow_stress(args, peak, args.steps, args.warmup, n_layers=80)
+    elif args.workload == "suffix":
+        out.update(suffix_transfers(args, peak, args.steps, args.warmup))
     elif args.workload == "compose":
         out["share"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=False)
         out["copy_all"] = compose_levels(args, peak, args.steps, args.warmup, copy_all=True)
@@ -776,7 +829,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=["8b", "8b-aligned", "70b", "8b-small", "tiny", "cow", "compose",
-                                                         "churn", "transfer", "meta", "costmodel"])
+                                                         "churn", "transfer", "meta", "costmodel", "suffix"])
     ap.add_argument("--block-size", type=int, default=16, help="churn workload only: 8, 16, 32 or 64")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 vector LD/ST per CTA, 2 cp.async.bulk, 3 vector LD/ST per warp")
     ap.add_argument("--min-seconds", type=float, default=1.0, help="repeat the timed region until this much device time is measured")
@@ -784,7 +837,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip roofline.per_workload (70B step, compose levels, COW stress)")
     args = ap.parse_args()
-    if args.workload in ("cow", "compose", "churn", "transfer", "meta", "costmodel"):
+    if args.workload in ("cow", "compose", "churn", "transfer", "meta", "costmodel", "suffix"):
         return extra_report(args)
     w = workload(args.workload)
     if args.impl == "reference":
@@ -837,6 +890,9 @@ def main():
             pw["compose_" + name] = lv
         pw["cow"] = cow_stress(args, peak, k, 2)
         pw["cow_70b"] = cow_stress(args, peak, k, 2, n_layers=80)
+        for name, rec in suffix_transfers(args, peak, k, 2).items():
+            if isinstance(rec, dict):
+                pw["suffix_" + name] = rec
         roofline["per_workload"] = pw
 
     if rank != 0:

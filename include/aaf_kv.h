@@ -173,6 +173,22 @@ int aaf_kv_materialize(aaf_kv_pool *pool, aaf_ctx_t ctx, int64_t tok_begin, int6
 int aaf_kv_import(aaf_kv_pool *pool, const void *src_dev, const aaf_kv_xfer_desc *desc, aaf_ctx_t *out_ctx,
                   void *stream);
 
+/* materialize / import, batched -- n independent transfers packed (unpacked) by one planner launch and ONE copy
+ * launch (Alg. "KV-Transfer": block selection by position range for several states at once; Sec. 5.4: only the
+ * subset a consumer needs is sent, so transfers are often short suffixes, whose copies are too small to reach the
+ * HBM rate one launch each).  When it succeeds the result is exactly that of the for-loop over i of
+ * aaf_kv_materialize(ctxs[i], tok_begin[i], tok_end[i], dst_dev[i], dst_bytes[i]) or of
+ * aaf_kv_import(src_dev[i], &descs[i]): the same handles (the n smallest free ones, in order), the same blocks
+ * (import i takes its blocks behind those of the imports before it), the same catalog stamps.  A context may
+ * appear in several entries of a materialize batch; destination buffers must not overlap.  All-or-nothing.
+ * All arrays are host arrays of n entries; out_descs may be NULL.  Errors: as the single forms, OOM_CTX /
+ * OOM_BLOCKS / TOO_MANY counted over the whole batch. */
+int aaf_kv_materialize_batch(aaf_kv_pool *pool, int32_t n, const aaf_ctx_t *ctxs, const int64_t *tok_begin,
+                             const int64_t *tok_end, void *const *dst_dev, const size_t *dst_bytes,
+                             aaf_kv_xfer_desc *out_descs, void *stream);
+int aaf_kv_import_batch(aaf_kv_pool *pool, int32_t n, const void *const *src_dev, const aaf_kv_xfer_desc *descs,
+                        aaf_ctx_t *out_ctxs, void *stream);
+
 /* fork -- Alg. "KV-Fork": k children alias the parent's blocks (table copied, refcount += 1 per
  * entry per child); nothing is copied, no block allocated (Sec. 3.3).  out_children (host, k
  * entries) receives the k smallest free handles in order.  Errors: BAD_CTX, INVALID_ARG, OOM_CTX,

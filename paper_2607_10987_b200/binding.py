@@ -73,6 +73,9 @@ SYMBOLS = {
     "aaf_kv_pool_destroy": (C.c_int, [_vp]),
     "aaf_kv_materialize": (C.c_int, [_vp, _i32, _i64, _i64, _vp, _sz, C.POINTER(aaf_kv_xfer_desc), _vp]),
     "aaf_kv_import": (C.c_int, [_vp, _vp, C.POINTER(aaf_kv_xfer_desc), _p32, _vp]),
+    "aaf_kv_materialize_batch": (C.c_int, [_vp, _i32, _p32, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_vp),
+                                           C.POINTER(_sz), C.POINTER(aaf_kv_xfer_desc), _vp]),
+    "aaf_kv_import_batch": (C.c_int, [_vp, _i32, C.POINTER(_vp), C.POINTER(aaf_kv_xfer_desc), _p32, _vp]),
     "aaf_kv_fork": (C.c_int, [_vp, _i32, _i32, _p32, _vp]),
     "aaf_kv_append": (C.c_int, [_vp, _i32, _p32, _p32, C.POINTER(_vp), _vp]),
     "aaf_kv_compose": (C.c_int, [_vp, _i32, _p32, _u32, _p32, _vp]),
@@ -137,6 +140,10 @@ def aaf_kv_pool_destroy(pool): return _fn("aaf_kv_pool_destroy")(pool)
 def aaf_kv_materialize(pool, ctx, t0, t1, dst, dst_bytes, out_desc, stream):
     return _fn("aaf_kv_materialize")(pool, ctx, t0, t1, dst, dst_bytes, out_desc, stream)
 def aaf_kv_import(pool, src, desc, out_ctx, stream): return _fn("aaf_kv_import")(pool, src, desc, out_ctx, stream)
+def aaf_kv_materialize_batch(pool, n, ctxs, t0, t1, dsts, dst_bytes, out_descs, stream):
+    return _fn("aaf_kv_materialize_batch")(pool, n, ctxs, t0, t1, dsts, dst_bytes, out_descs, stream)
+def aaf_kv_import_batch(pool, n, srcs, descs, out_ctxs, stream):
+    return _fn("aaf_kv_import_batch")(pool, n, srcs, descs, out_ctxs, stream)
 def aaf_kv_fork(pool, parent, k, out_children, stream): return _fn("aaf_kv_fork")(pool, parent, k, out_children, stream)
 def aaf_kv_append(pool, n, ctxs, n_new, srcs, stream): return _fn("aaf_kv_append")(pool, n, ctxs, n_new, srcs, stream)
 def aaf_kv_compose(pool, m, segs, flags, out_ctx, stream): return _fn("aaf_kv_compose")(pool, m, segs, flags, out_ctx, stream)
@@ -276,6 +283,25 @@ class KVPool:
         out = C.c_int32(-1)
         st = aaf_kv_import(self.h, buf.data_ptr(), C.byref(xd), C.byref(out), self._stream())
         return st, (out.value if st == AAF_OK else None)
+
+    def materialize_batch(self, ctxs, t0s, t1s, outs):
+        """outs: one device tensor per entry.  Returns the status."""
+        n = len(ctxs)
+        a = (C.c_int32 * max(n, 1))(*ctxs)
+        b0 = (C.c_int64 * max(n, 1))(*t0s)
+        b1 = (C.c_int64 * max(n, 1))(*t1s)
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in outs])
+        sizes = (C.c_size_t * max(n, 1))(*[t.numel() * t.element_size() for t in outs])
+        return aaf_kv_materialize_batch(self.h, n, a, b0, b1, ptrs, sizes, None, self._stream())
+
+    def import_batch(self, bufs, ns):
+        """bufs: one device transfer buffer per entry, ns: its token count.  Returns (status, [handles])."""
+        n = len(bufs)
+        ptrs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in bufs])
+        descs = (aaf_kv_xfer_desc * max(n, 1))(*[self.xfer_desc(k) for k in ns])
+        out = (C.c_int32 * max(n, 1))()
+        st = aaf_kv_import_batch(self.h, n, ptrs, descs, out, self._stream())
+        return st, (list(out[:n]) if st == AAF_OK else None)
 
     def fork(self, parent, k):
         out = (C.c_int32 * max(k, 1))()

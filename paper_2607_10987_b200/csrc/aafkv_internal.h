@@ -100,6 +100,22 @@ struct ComposeSeg {       // 56 bytes; one per segment of every merge of a batch
     int first_ctx;        // last segment of a result only: handle of the result's first segment, else -1
 };
 static_assert(sizeof(ComposeSeg) == 56, "ComposeSeg layout");
+struct MatEntry {         // 40 bytes; one token range of one context gathered into one transfer buffer
+    char *dst;            // device transfer buffer of t1 - t0 tokens
+    long long t0, t1;     // token range
+    int ctx;
+    int piece_off;        // first piece slot of the entry: one piece per block of the range
+    int out_index;        // position in the batch (its logical clock is the call's clock + out_index)
+    int table_j0;         // table position held by the first entry of the context's table row (0 for a pool)
+};
+struct ImpEntry {         // 32 bytes; one transfer buffer registered as one new context
+    const char *src;      // device transfer buffer of n tokens
+    long long n;
+    int ctx;              // handle of the new context
+    int block_off;        // rank (from the ring head, over the batch) of its first block = its first piece slot
+    int out_index;
+    int pad;
+};
 struct EvictArgs {        // followed by int ctx[n], int ent_off[n + 1]
     int n;
     int total;
@@ -117,12 +133,24 @@ struct SmallAppend {
 struct SmallCompose {
     ComposeSeg s[SMALL_RECORDS];
 };
+struct SmallMat {
+    MatEntry e[SMALL_RECORDS];
+};
+struct SmallImp {
+    ImpEntry e[SMALL_RECORDS];
+};
 
 // ---- launchers (each returns cudaGetLastError() of its launches)
 // `clock` is the logical clock of the call (count of successful state-touching calls); planners stamp
 // it into the catalog.  A DevState without catalog arrays (cat_len == nullptr) skips the stamping.
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
                                     long long clock, cudaStream_t st, int table_j0 = 0);
+// batched forms: ents_dev == nullptr means the n <= SMALL_RECORDS records are in `small`; entry i is stamped clock + i
+cudaError_t launch_plan_materialize_batch(const Geom &g, const DevState &s, const MatEntry *ents_dev,
+                                          const SmallMat &small, int n, int total_pieces, long long clock,
+                                          cudaStream_t st);
+cudaError_t launch_plan_import_batch(const Geom &g, const DevState &s, const ImpEntry *ents_dev, const SmallImp &small,
+                                     int n, int total_blocks, long long clock, cudaStream_t st);
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
                                long long clock, cudaStream_t st);
 // children_dev == nullptr: the k <= SMALL_ARGS children are in `small`

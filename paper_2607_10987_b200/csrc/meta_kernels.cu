@@ -126,64 +126,102 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *total) {
 }
 
 // ------------------------------------------------------------------------------------------
-// materialize: one piece per block of the token range
-// `table_j0`: table position held by the first entry of the context's table row (0 for a pool; a caller that
-// uploads only the slice of a table it needs passes the slice's first position)
-__global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState s, int ctx, long long t0,
-                                                               long long t1, char *dst, long long clock,
-                                                               int table_j0) {
-    const long long j0 = t0 / g.BS, j1 = (t1 - 1) / g.BS;
-    const long long n = t1 - t0;
-    const int *table = s.tables + (long long)ctx * g.max_blk;
-    for (long long j = j0 + blockIdx.x * blockDim.x + threadIdx.x; j <= j1; j += (long long)gridDim.x * blockDim.x) {
-        const long long lo = max(t0, j * g.BS), hi = min(t1, (j + 1) * g.BS);
-        const int b = table[j - table_j0];
-        if (b < 0 || b >= g.NB) {  // never gather through an entry that does not name a pool block
-            clear_piece(s.pieces[j - j0]);
-            set_status(s.ctl, AAF_ERR_CORRUPT, 10);
-            continue;
-        }
-        s.pieces[j - j0] = make_piece(pool_slot(g, b, lo - j * g.BS), g.layer_stride, g.run, dst + (lo - t0) * g.row,
-                                      2 * n * g.row, n * g.row, (unsigned)((hi - lo) * g.row));
+// last record whose first slot is <= sl (records sorted by their first slot)
+template <typename T, typename F>
+__device__ __forceinline__ int find_record(const T *rec, int n, int sl, F first_slot) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (first_slot(rec[mid]) <= sl) lo = mid; else hi = mid - 1;
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(n * 2 * g.L * g.row));
-        if (s.cat_len) {  // the state was read by a transfer
-            s.cat_reuse[ctx] += 1;
-            s.cat_last[ctx] = clock;
-        }
-    }
+    return lo;
 }
 
 // ------------------------------------------------------------------------------------------
-// import: reserve ceil(n / BS) ring entries in order, write the table, one piece per block
-__global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevState s, int ctx, long long n,
-                                                                   const char *src, long long clock) {
-    const int nblk = (int)((n + g.BS - 1) / g.BS);
-    const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
-    const bool ok = (tail - head0) >= (unsigned long long)nblk;
-    int *table = s.tables + (long long)ctx * g.max_blk;
-    for (int j = threadIdx.x; j < nblk; j += blockDim.x) {
-        if (!ok) {
-            clear_piece(s.pieces[j]);
+// materialize: one piece per block of every token range of the batch.  A pure read of the pool, so a batch is
+// the loop over its entries in any order; the catalog is stamped as the loop would stamp it.
+constexpr int MAT_STAGE = 512;
+__global__ void __launch_bounds__(256) plan_materialize_kernel(Geom g, DevState s,
+                                                               const MatEntry *__restrict__ ents_host, SmallMat small,
+                                                               int n, int total_pieces, long long clock) {
+    __shared__ MatEntry sh_ent[MAT_STAGE];
+    const MatEntry *ent;
+    if (ents_host) {
+        ent = stage_args(ents_host, n, sh_ent, MAT_STAGE);
+    } else {  // a small batch arrives as kernel parameters
+        if (threadIdx.x < n) sh_ent[threadIdx.x] = small.e[threadIdx.x];
+        __syncthreads();
+        ent = sh_ent;
+    }
+    for (int sl = blockIdx.x * blockDim.x + threadIdx.x; sl < total_pieces; sl += gridDim.x * blockDim.x) {
+        const MatEntry e = ent[find_record(ent, n, sl, [](const MatEntry &r) { return r.piece_off; })];
+        const long long cnt = e.t1 - e.t0;
+        const long long j = e.t0 / g.BS + (sl - e.piece_off);  // table position of the block
+        const long long lo = max(e.t0, j * g.BS), hi = min(e.t1, (j + 1) * g.BS);
+        const int b = s.tables[(long long)e.ctx * g.max_blk + (j - e.table_j0)];
+        if (b < 0 || b >= g.NB) {  // never gather through an entry that does not name a pool block
+            clear_piece(s.pieces[sl]);
+            set_status(s.ctl, AAF_ERR_CORRUPT, 10);
             continue;
         }
-        const int b = ring_at(s.ring, head0 + j, g.NB);
-        claim_block(s, b, g.NB);
-        table[j] = b;
-        const long long lo = (long long)j * g.BS, hi = min(n, lo + g.BS);
-        s.pieces[j] = make_piece(src + lo * g.row, 2 * n * g.row, n * g.row, pool_slot(g, b, 0), g.layer_stride, g.run,
-                                 (unsigned)((hi - lo) * g.row));
+        s.pieces[sl] = make_piece(pool_slot(g, b, lo - j * g.BS), g.layer_stride, g.run, e.dst + (lo - e.t0) * g.row,
+                                  2 * cnt * g.row, cnt * g.row, (unsigned)((hi - lo) * g.row));
     }
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            atomicAdd(&s.ctl->payload_bytes, (unsigned long long)((ent[i].t1 - ent[i].t0) * 2 * g.L * g.row));
+            if (s.cat_len) {  // the state was read by a transfer
+                atomicAdd(&s.cat_reuse[ent[i].ctx], 1ull);
+                atomicMax(&s.cat_last[ent[i].ctx], clock + ent[i].out_index);
+            }
+        }
+}
+
+// ------------------------------------------------------------------------------------------
+// import: one ring reservation for the whole batch; entry i takes ceil(n_i / BS) entries behind those of the
+// entries before it (what the loop over the batch would take), writes its table, one piece per block
+constexpr int IMP_STAGE = 512;
+__global__ void __launch_bounds__(PLAN_THREADS) plan_import_kernel(Geom g, DevState s,
+                                                                   const ImpEntry *__restrict__ ents_host,
+                                                                   SmallImp small, int n, int total_blocks,
+                                                                   long long clock) {
+    __shared__ ImpEntry sh_ent[IMP_STAGE];
+    const ImpEntry *ent;
+    if (ents_host) {
+        ent = stage_args(ents_host, n, sh_ent, IMP_STAGE);
+    } else {  // a small batch arrives as kernel parameters
+        if (threadIdx.x < n) sh_ent[threadIdx.x] = small.e[threadIdx.x];
+        __syncthreads();
+        ent = sh_ent;
+    }
+    const unsigned long long head0 = s.ctl->head, tail = s.ctl->tail;
+    const bool ok = (tail - head0) >= (unsigned long long)total_blocks;
+    for (int sl = threadIdx.x; sl < total_blocks; sl += blockDim.x) {
+        if (!ok) {
+            clear_piece(s.pieces[sl]);
+            continue;
+        }
+        const ImpEntry e = ent[find_record(ent, n, sl, [](const ImpEntry &r) { return r.block_off; })];
+        const int j = sl - e.block_off;
+        const int b = ring_at(s.ring, head0 + (unsigned long long)sl, g.NB);
+        claim_block(s, b, g.NB);
+        s.tables[(long long)e.ctx * g.max_blk + j] = b;
+        const long long lo = (long long)j * g.BS, hi = min(e.n, lo + g.BS);
+        s.pieces[sl] = make_piece(e.src + lo * g.row, 2 * e.n * g.row, e.n * g.row, pool_slot(g, b, 0), g.layer_stride,
+                                  g.run, (unsigned)((hi - lo) * g.row));
+    }
+    if (ok)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            atomicAdd(&s.ctl->payload_bytes, (unsigned long long)(ent[i].n * 2 * g.L * g.row));
+            if (s.cat_len) catalog_born(s, ent[i].ctx, ent[i].n, clock + ent[i].out_index, 1, -1);
+        }
     __syncthreads();  // every thread has read head0 before it moves
     if (threadIdx.x == 0) {
         if (!ok) {
             set_status(s.ctl, AAF_ERR_CORRUPT, 3);
         } else {
-            s.ctl->head = head0 + nblk;
-            note_alloc(s.ctl, g, head0 + nblk, tail);
-            s.ctl->payload_bytes += (unsigned long long)(n * 2 * g.L * g.row);
-            if (s.cat_len) catalog_born(s, ctx, n, clock, 1, -1);
+            s.ctl->head = head0 + total_blocks;
+            note_alloc(s.ctl, g, head0 + total_blocks, tail);
         }
     }
 }
@@ -815,16 +853,29 @@ static int grid_for(long long items, int threads, int cap) {
     return (int)gsz;
 }
 
+cudaError_t launch_plan_materialize_batch(const Geom &g, const DevState &s, const MatEntry *ents_dev,
+                                          const SmallMat &small, int n, int total_pieces, long long clock,
+                                          cudaStream_t st) {
+    plan_materialize_kernel<<<grid_for(total_pieces, 256, 64), 256, 0, st>>>(g, s, ents_dev, small, n, total_pieces,
+                                                                              clock);
+    return cudaGetLastError();
+}
 cudaError_t launch_plan_materialize(const Geom &g, const DevState &s, int ctx, long long t0, long long t1, char *dst,
                                     long long clock, cudaStream_t st, int table_j0) {
-    const long long nb = (t1 - 1) / g.BS - t0 / g.BS + 1;
-    plan_materialize_kernel<<<grid_for(nb, 256, 64), 256, 0, st>>>(g, s, ctx, t0, t1, dst, clock, table_j0);
+    SmallMat one{};
+    one.e[0].dst = dst; one.e[0].t0 = t0; one.e[0].t1 = t1; one.e[0].ctx = ctx; one.e[0].table_j0 = table_j0;
+    return launch_plan_materialize_batch(g, s, nullptr, one, 1, (int)((t1 - 1) / g.BS - t0 / g.BS + 1), clock, st);
+}
+cudaError_t launch_plan_import_batch(const Geom &g, const DevState &s, const ImpEntry *ents_dev, const SmallImp &small,
+                                     int n, int total_blocks, long long clock, cudaStream_t st) {
+    plan_import_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, ents_dev, small, n, total_blocks, clock);
     return cudaGetLastError();
 }
 cudaError_t launch_plan_import(const Geom &g, const DevState &s, int ctx, long long n, const char *src,
                                long long clock, cudaStream_t st) {
-    plan_import_kernel<<<1, PLAN_THREADS, 0, st>>>(g, s, ctx, n, src, clock);
-    return cudaGetLastError();
+    SmallImp one{};
+    one.e[0].src = src; one.e[0].n = n; one.e[0].ctx = ctx;
+    return launch_plan_import_batch(g, s, nullptr, one, 1, (int)((n + g.BS - 1) / g.BS), clock, st);
 }
 cudaError_t launch_fork(const Geom &g, const DevState &s, int parent, long long T, int k, const int *children_dev,
                         const SmallInts &small, long long clock, cudaStream_t st) {

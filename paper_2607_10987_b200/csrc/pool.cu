@@ -40,6 +40,10 @@ using namespace aafkv;
 namespace {
 
 constexpr int ARG_SLOTS = 16;
+constexpr size_t ARG_RECORD_BYTES = 64;  // per-record room in a slot of the pinned argument ring
+static_assert(sizeof(ComposeSeg) <= ARG_RECORD_BYTES && sizeof(AppendEntry) <= ARG_RECORD_BYTES &&
+                  sizeof(MatEntry) <= ARG_RECORD_BYTES && sizeof(ImpEntry) <= ARG_RECORD_BYTES,
+              "argument records must fit their room in the pinned ring");
 
 struct Layout {
     size_t ctl, refcount, ring, last_pos, tables, pieces, scratch, cat_len, cat_reuse, cat_last, cat_score, cat_origin, cat_parent, cat_born, cat_parent_born, tile_count, total;
@@ -467,7 +471,7 @@ int aaf_kv_pool_create(const aaf_kv_pool_desc *desc, aaf_kv_pool **out) {
 
     bool ok = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) == cudaSuccess;
     ok = ok && copy_tuning_init(p->g.run, &p->tuning) == cudaSuccess;
-    p->slot_bytes = align_up(48 * (size_t)lay.max_batch + 256, 256);
+    p->slot_bytes = align_up(ARG_RECORD_BYTES * (size_t)lay.max_batch + 256, 256);
     ok = ok && cudaHostAlloc(reinterpret_cast<void **>(&p->args), p->slot_bytes * ARG_SLOTS, cudaHostAllocMapped) ==
                    cudaSuccess;
     for (int i = 0; ok && i < ARG_SLOTS; ++i)
@@ -567,6 +571,103 @@ int aaf_kv_import(aaf_kv_pool *p, const void *src_dev, const aaf_kv_xfer_desc *d
     if (p->broken) return AAF_ERR_CUDA;
     DeviceGuard guard(p->device);
     return import_impl(p, src_dev, desc, out_ctx, static_cast<cudaStream_t>(stream), nullptr);
+}
+
+int aaf_kv_materialize_batch(aaf_kv_pool *p, int32_t n, const aaf_ctx_t *ctxs, const int64_t *tok_begin,
+                             const int64_t *tok_end, void *const *dst_dev, const size_t *dst_bytes,
+                             aaf_kv_xfer_desc *out_descs, void *stream) {
+    AAF_RANGE("aaf_kv_materialize_batch");
+    if (!p || n < 1 || !ctxs || !tok_begin || !tok_end || !dst_dev || !dst_bytes) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
+    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    long long slots = 0, tokens = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!is_live(p, ctxs[i])) return AAF_ERR_BAD_CTX;
+        const long long t0 = tok_begin[i], t1 = tok_end[i];
+        if (!aligned16(dst_dev[i]) || t0 < 0 || t0 >= t1 || t1 > p->len[ctxs[i]]) return AAF_ERR_INVALID_ARG;
+        if ((unsigned long long)dst_bytes[i] < (unsigned long long)((t1 - t0) * bpt_of(p))) return AAF_ERR_DST_TOO_SMALL;
+        slots += (t1 - 1) / p->g.BS - t0 / p->g.BS + 1;
+        tokens += t1 - t0;
+    }
+    if (slots > p->lay.max_pieces) return AAF_ERR_TOO_MANY;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    // a small batch travels as kernel parameters, a large one through the pinned argument ring
+    SmallMat small{};
+    const bool by_value = n <= SMALL_RECORDS;
+    MatEntry *ent = by_value ? small.e : reinterpret_cast<MatEntry *>(acquire_args(p));
+    int off = 0;
+    for (int i = 0; i < n; ++i) {
+        MatEntry &e = ent[i];
+        e.dst = static_cast<char *>(dst_dev[i]);
+        e.t0 = tok_begin[i]; e.t1 = tok_end[i];
+        e.ctx = ctxs[i]; e.piece_off = off; e.out_index = i; e.table_j0 = 0;
+        off += (int)((e.t1 - 1) / p->g.BS - e.t0 / p->g.BS + 1);
+    }
+    const PlanSlot ps = begin_plan(p);
+    const cudaError_t e = launch_plan_materialize_batch(p->g, ps.view, by_value ? nullptr : ent, small, n, (int)slots,
+                                                        p->clock + 1, p->meta_stream);
+    if (!by_value) release_args(p, p->meta_stream);
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
+    p->clock += n;  // entry i of the batch is the call with clock + 1 + i
+    p->meta_launches += 1;
+    const int rc = run_copy(p, ps, AAF_OP_MATERIALIZE, (int)slots, tokens, st);
+    end_copy(p, ps, st);
+    if (rc == AAF_OK && out_descs)
+        for (int i = 0; i < n; ++i) fill_desc(p, &out_descs[i], tok_begin[i], tok_end[i] - tok_begin[i]);
+    return rc;
+}
+
+int aaf_kv_import_batch(aaf_kv_pool *p, int32_t n, const void *const *src_dev, const aaf_kv_xfer_desc *descs,
+                        aaf_ctx_t *out_ctxs, void *stream) {
+    AAF_RANGE("aaf_kv_import_batch");
+    if (!p || n < 1 || !src_dev || !descs || !out_ctxs) return AAF_ERR_INVALID_ARG;
+    if (p->broken) return AAF_ERR_CUDA;
+    if (n > p->lay.max_batch) return AAF_ERR_TOO_MANY;
+    long long blocks = 0, tokens = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!aligned16(src_dev[i])) return AAF_ERR_INVALID_ARG;
+        if (!compatible(p, &descs[i])) return AAF_ERR_INCOMPAT;
+        if (descs[i].n_tokens < 1) return AAF_ERR_INVALID_ARG;
+        if (nblk_of(p, descs[i].n_tokens) > p->g.max_blk) return AAF_ERR_TOO_LONG;
+        blocks += nblk_of(p, descs[i].n_tokens);
+        tokens += descs[i].n_tokens;
+    }
+    if (blocks > p->lay.max_pieces) return AAF_ERR_TOO_MANY;
+    if (p->g.max_ctx - p->live_ctx < n) return AAF_ERR_OOM_CTX;
+    DeviceGuard guard(p->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int rc0 = ensure_free(p, blocks, st);
+    if (rc0 != AAF_OK) return rc0;
+    p->last_stream = st;
+    SmallImp small{};
+    const bool by_value = n <= SMALL_RECORDS;
+    ImpEntry *ent = by_value ? small.e : reinterpret_cast<ImpEntry *>(acquire_args(p));
+    int c = -1, off = 0;
+    for (int i = 0; i < n; ++i) {  // the n smallest free handles, in order: what the loop of imports would take
+        c = smallest_free_ctx(p, c + 1);
+        ImpEntry &e = ent[i];
+        e.src = static_cast<const char *>(src_dev[i]);
+        e.n = descs[i].n_tokens;
+        e.ctx = c; e.block_off = off; e.out_index = i; e.pad = 0;
+        off += (int)nblk_of(p, e.n);
+    }
+    const PlanSlot ps = begin_plan(p);
+    const cudaError_t e = launch_plan_import_batch(p->g, ps.view, by_value ? nullptr : ent, small, n, (int)blocks,
+                                                   p->clock + 1, p->meta_stream);
+    // the handles are read back from the records before the ring slot is released
+    for (int i = 0; i < n; ++i) out_ctxs[i] = ent[i].ctx;
+    if (!by_value) release_args(p, p->meta_stream);
+    if (e != cudaSuccess || !end_plan(p, ps, st)) return broke(p);
+    p->clock += n;
+    p->meta_launches += 1;
+    p->free_lb -= blocks;
+    for (int i = 0; i < n; ++i) p->len[out_ctxs[i]] = descs[i].n_tokens;
+    p->live_ctx += n;
+    const int rc = run_copy(p, ps, AAF_OP_IMPORT, (int)blocks, tokens, st);
+    end_copy(p, ps, st);
+    return rc;
 }
 
 int aaf_kv_import_host(aaf_kv_pool *p, const void *src_host, const aaf_kv_xfer_desc *desc, void *staging_dev,

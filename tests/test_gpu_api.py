@@ -320,7 +320,8 @@ def test_default_bench_line_carries_the_other_full_size_workloads():
     d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
     assert d["config"]["n_blocks"] == 32768 and d["gpu_launches"] == 3 * 12
     pw = d["roofline"]["per_workload"]
-    assert set(pw) == {"70b", "compose_pairs", "compose_quads", "compose_all16", "compose_flat16", "cow", "cow_70b"}
+    assert set(pw) == {"70b", "compose_pairs", "compose_quads", "compose_all16", "compose_flat16", "cow", "cow_70b",
+                       "suffix_pack_loop", "suffix_pack_batch", "suffix_unpack_loop", "suffix_unpack_batch"}
     for name, rec in pw.items():
         assert set(rec) >= {"achieved", "frac", "algorithmic_bytes_per_launch", "mean_launch_ms", "launches"}, name
         assert 0.5 < rec["frac"] < 1.2 and rec["launches"] > 0, (name, rec["frac"])

@@ -495,3 +495,85 @@ def test_compose_batch_is_all_or_nothing():
     assert gpu.o.compose_batch([[0, 3]], configs.COMPOSE_COPY_ALL) == (0, [4])
     assert cpu.compose([0, 3], configs.COMPOSE_COPY_ALL) == (0, 4)
     assert gpu.snapshot() == cpu.snapshot() and gpu.o.sync_status() == 0
+
+
+def test_batches_at_the_batch_limit_go_through_the_argument_ring():
+    """1000 segments in one merge, 1000 merges in one batch, 1000 transfers in one batch: the records travel
+    through the pinned argument ring (not as kernel parameters) and must fit it."""
+    g = Geometry(2, 1, 8, 16, 2, 4096, 1030, 800)  # 16-byte rows
+    seed = 41
+    order = configs.free_order(seed, g.n_blocks)
+    gpu = GpuBackend(g, seed, free_order=order)
+    cpu = OracleBackend(g, seed, free_order=order)
+    for be in (gpu, cpu):
+        assert be.imp(be.payload(seed, 1, 3), 3) == (0, 0)
+        assert be.imp(be.payload(seed, 2, 21), 21) == (0, 1)
+    # one merge of 1000 segments
+    segs = [0, 1] * 500
+    assert gpu.compose(segs, 0) == cpu.compose(segs, 0) == (0, 2)
+    assert gpu.snapshot() == cpu.snapshot()
+    # 1000 merges of one or two segments in one batch, 1024 segments in all (results 3 .. 1002)
+    batch = [[1, 0] if i < 24 else [i % 3] for i in range(1000)]
+    st, outs = gpu.o.compose_batch(batch, 0)
+    assert st == 0 and outs == list(range(3, 1003))
+    for b in batch:
+        assert cpu.compose(b, 0)[0] == 0
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.catalog() == cpu.o.catalog()
+    # 1000 gathers in one batch, compared with the oracle's loop
+    import torch
+
+    ctxs = [3 + i for i in range(1000)]
+    lens = [min(cpu.o.ctx_len(c), 20) for c in ctxs]  # the first 20 tokens of each: at most two blocks per entry
+    outs_dev = [torch.empty(n * g.bpt, dtype=torch.uint8, device=gpu.o.device) for n in lens]
+    assert gpu.o.materialize_batch(ctxs, [0] * 1000, lens, outs_dev) == 0
+    for c, n, d in zip(ctxs, lens, outs_dev):
+        st, want = cpu.materialize(c, 0, n)
+        assert st == 0 and np.array_equal(d.cpu().numpy(), want), c
+    assert gpu.o.catalog() == cpu.o.catalog()
+    assert np.array_equal(gpu.pool_layers(range(g.n_layers)), cpu.o.pool_view())
+    assert gpu.o.sync_status() == 0
+
+
+def test_materialize_and_import_batches_equal_the_loops():
+    """aaf_kv_materialize_batch / aaf_kv_import_batch against the oracle's loops of single calls: ragged ranges,
+    a context gathered twice, block tables and handles of the imported batch, catalog stamps, one copy launch each."""
+    import torch
+
+    from paper_2607_10987_b200 import binding
+
+    lens = [37, 64, 16, 5, 100, 48, 33, 1, 80, 250]
+    g, gpu, cpu = _merge_pool(33, lens)
+    dev = gpu.o.device
+    ranges = [(0, 0, 37), (1, 16, 64), (4, 3, 99), (9, 17, 250), (4, 0, 100), (7, 0, 1), (3, 2, 5), (8, 79, 80),
+              (2, 0, 16), (5, 15, 17)]
+    outs = [torch.full(((b - a) * g.bpt,), 0xEE, dtype=torch.uint8, device=dev) for _, a, b in ranges]
+    l0 = gpu.o.stats()["copy_launches"]["materialize"]
+    assert gpu.o.materialize_batch([c for c, _, _ in ranges], [a for _, a, _ in ranges], [b for _, _, b in ranges],
+                                   outs) == 0
+    assert gpu.o.stats()["copy_launches"]["materialize"] == l0 + 1
+    want = []
+    for (c, a, b), d in zip(ranges, outs):
+        st, w = cpu.materialize(c, a, b)
+        assert st == 0 and np.array_equal(d.cpu().numpy(), w), (c, a, b)
+        want.append(w)
+    assert gpu.o.catalog() == cpu.o.catalog()
+    # register all ten buffers as new contexts in one call
+    st, new = gpu.o.import_batch(outs, [b - a for _, a, b in ranges])
+    assert st == 0 and gpu.o.stats()["copy_launches"]["import"] == len(lens) + 1
+    for w, (c, a, b), h in zip(want, ranges, new):
+        assert cpu.imp(w, b - a) == (0, h)
+    assert gpu.snapshot() == cpu.snapshot() and gpu.o.catalog() == cpu.o.catalog()
+    same_catalog_export(gpu, cpu)
+    assert np.array_equal(gpu.pool_layers(range(g.n_layers)), cpu.o.pool_view())
+    # all-or-nothing
+    before = gpu.snapshot()
+    small = torch.empty(16, dtype=torch.uint8, device=dev)
+    assert gpu.o.materialize_batch([0, 1], [0, 0], [37, 64], [outs[0], small]) == binding.AAF_ERR_DST_TOO_SMALL
+    assert gpu.o.materialize_batch([0, 39], [0, 0], [37, 1], [outs[0], outs[5]]) == binding.AAF_ERR_BAD_CTX
+    assert gpu.o.materialize_batch([0, 1], [0, 0], [37, 65], [outs[0], outs[1]]) == binding.AAF_ERR_INVALID_ARG
+    big = [gpu.payload(33, 50, 1500)] * 5
+    assert gpu.o.stats()["free_blocks"] < 5 * 94
+    assert gpu.o.import_batch(big, [1500] * 5)[0] == binding.AAF_ERR_OOM_BLOCKS  # 5 x 94 blocks, fewer are free
+    assert gpu.o.import_batch([big[0]], [1600])[0] == binding.AAF_ERR_TOO_LONG     # 100 blocks > 96
+    assert gpu.o.import_batch([outs[0]] * 25, [37] * 25)[0] == binding.AAF_ERR_OOM_CTX  # 40 handles, 20 live
+    assert gpu.snapshot() == before and gpu.o.catalog() == cpu.o.catalog() and gpu.o.sync_status() == 0
