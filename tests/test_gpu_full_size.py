@@ -229,6 +229,36 @@ def test_config2_host_buffer_path_value_model_all_layers():
     assert pool.sync_status() == 0 and pool.stats()["cow_count"] == 2 * agents
 
 
+def test_suffix_transfer_batches_value_model_all_layers():
+    """Batched partial transfers at the 8B shape on the full pool: the 512-token continuations of 16 agents packed by
+    one aaf_kv_materialize_batch call and registered by one aaf_kv_import_batch call; every buffer and every live
+    context compared in all layers with the value model."""
+    import torch
+
+    from tests.value_check import Paired
+
+    g, seed, _ = configs.config2(True)
+    if not _fits(g, 12):
+        pytest.skip("not enough free device memory for the 64 GiB pool")
+    T, agents, n_new = 8187, 16, 512
+    gpu = GpuBackend(g, seed, free_order=configs.free_order(seed, g.n_blocks), init_fill=False)
+    sh = ShadowBackend(gpu)
+    st, root = sh.imp(sh.payload(seed, 1, T), T)
+    st, kids = sh.fork(root, agents)
+    assert sh.append(kids, [n_new] * agents, [sh.payload(seed, 2 + i, n_new) for i in range(agents)])[0] == 0
+    bufs = [torch.empty(n_new * g.bpt, dtype=torch.uint8, device=gpu.o.device) for _ in range(agents)]
+    assert gpu.o.materialize_batch(kids, [T] * agents, [T + n_new] * agents, bufs) == 0
+    seqs = [sh.vm.materialize(k, T, T + n_new) for k in kids]
+    for b, seq in zip(bufs, seqs):
+        sh.check_buffer(seed, Paired(b, seq))
+    st, new = gpu.o.import_batch(bufs, [n_new] * agents)
+    assert st == 0
+    assert [sh.vm.imp(seq) for seq in seqs] == new
+    sh.check_all_live(seed)
+    check_conservation(gpu.snapshot(), g.n_blocks, g.block_size)
+    assert gpu.o.sync_status() == 0 and len(sh.vm.ctx) == 1 + 2 * agents
+
+
 def test_config4_llama70b_value_model_all_layers():
     g, seed, ops = configs.config4(True)
     if not _fits(g, 40):
