@@ -100,6 +100,32 @@ int main(void) {
     encode(want, root_ids, 6);
     if (memcmp(host, want, 6 * BPT) != 0) { fprintf(stderr, "parent changed\n"); return 8; }
 
+    /* batched calls from C: two merges in one call, then both results gathered by one call into one buffer each */
+    {
+        const int32_t seg_off[3] = {0, 2, 3};
+        const aaf_ctx_t bsegs[3] = {kids[1], kids[0], root}; /* merge 0 = child 1 || child 0, merge 1 = root alone */
+        aaf_ctx_t outs[2] = {-1, -1};
+        CHECK(aaf_kv_compose_batch(pool, 2, seg_off, bsegs, AAF_COMPOSE_SHARE, outs, st));
+        const int64_t b0[2] = {0, 2}, b1[2] = {15, 6};
+        void *dsts[2] = {dev_out, dev_out + 16 * BPT};
+        const size_t caps[2] = {15 * BPT, 4 * BPT};
+        CHECK(aaf_kv_materialize_batch(pool, 2, outs, b0, b1, dsts, caps, NULL, st));
+        cudaMemcpyAsync(host, dev_out, 32 * BPT, cudaMemcpyDeviceToHost, st);
+        cudaStreamSynchronize(st);
+        int m0[15] = {0, 1, 2, 3, 4, 5, 0, 1, 2, 3, 4, 5, 100, 101, 102}, m1[4] = {2, 3, 4, 5};
+        encode(want, m0, 15);
+        if (memcmp(host, want, 15 * BPT) != 0) { fprintf(stderr, "batched merge 0 differs\n"); return 12; }
+        encode(want, m1, 4);
+        if (memcmp(host + 16 * BPT, want, 4 * BPT) != 0) { fprintf(stderr, "batched gather 1 differs\n"); return 13; }
+        /* register both buffers as new contexts in one call, then drop the four batch products again */
+        const void *srcs2[2] = {dev_out, dev_out + 16 * BPT};
+        aaf_kv_xfer_desc xds[2] = {{7, 9, L, H, D, E, 0, 15}, {7, 9, L, H, D, E, 2, 4}};
+        aaf_ctx_t regs[2] = {-1, -1};
+        CHECK(aaf_kv_import_batch(pool, 2, srcs2, xds, regs, st));
+        aaf_ctx_t drop[4] = {outs[0], outs[1], regs[0], regs[1]};
+        CHECK(aaf_kv_evict(pool, 4, drop, st));
+    }
+
     /* reference counts are conserved; evicting everything returns every block */
     int32_t rc[NB], fl[NB], nfree = 0, sum = 0;
     CHECK(aaf_kv_get_refcounts(pool, rc));

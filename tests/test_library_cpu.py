@@ -81,3 +81,9 @@ def test_strerror_names_every_status():
 def test_null_pool_is_rejected():
     assert binding.aaf_kv_evict(None, 1, (C.c_int32 * 1)(0), None) == binding.AAF_ERR_INVALID_ARG
     assert binding.aaf_kv_sync_status(None) == binding.AAF_ERR_INVALID_ARG
+    one = (C.c_int32 * 2)(0, 1)
+    assert binding.aaf_kv_compose_batch(None, 1, one, one, 0, one, None) == binding.AAF_ERR_INVALID_ARG
+    assert binding.aaf_kv_materialize_batch(None, 1, one, None, None, None, None, None, None) == \
+        binding.AAF_ERR_INVALID_ARG
+    assert binding.aaf_kv_import_batch(None, 1, None, None, one, None) == binding.AAF_ERR_INVALID_ARG
+    assert binding.aaf_kv_append_host(None, 1, one, one, None, None, 0, None) == binding.AAF_ERR_INVALID_ARG
