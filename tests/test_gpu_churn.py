@@ -156,7 +156,8 @@ def test_full_size_trace_8b_pool_metadata_against_small_row_oracle():
     assert gs["payload_bytes"] == cs["rows_copied"] * g.row * g.n_layers  # same rows moved, full-size bytes
 
 
-def test_full_size_trace_8b_pool_value_model_all_layers():
+@pytest.mark.parametrize("bs", [8, 16, 32, 64])
+def test_full_size_trace_8b_pool_value_model_all_layers(bs):
     """The benchmark-sized trace (8B rows, 32 layers, pool = 75 % of demand, about 60 GiB) with the value model
     beside the library instead of the paged oracle: no block id, free-list order or reference count is
     compared, only what the operators MEAN.  Every 5th materialised buffer and, at the end, every live context
@@ -166,7 +167,7 @@ def test_full_size_trace_8b_pool_value_model_all_layers():
 
     import torch
 
-    bs, cap = 16, 32768
+    cap = 32768
     small = lambda nb: Geometry(1, 1, 8, bs, 2, nb, 80, cap // bs)
     demand = demand_blocks(small, cap, bs, 10000)
     nb = int(0.75 * demand)
