@@ -410,6 +410,11 @@ int aaf_kv_materialize_noalloc(const void *pool_base_dev, size_t layer_stride_by
  * AAF_ERR_TIMEOUT once, and the pool keeps working.  Nothing faults, traps or hangs. */
 int aaf_kv_debug_expire_wait(aaf_kv_pool *pool, uint64_t limit_cycles, void *stream);
 
+/* Test hook for the error contract (no paper counterpart): puts the pool into the state that a CUDA runtime failure
+ * inside an operator leaves it in, without any failure.  Every later operator call then returns AAF_ERR_CUDA and
+ * changes nothing; introspection and aaf_kv_pool_destroy keep working. */
+int aaf_kv_debug_mark_unusable(aaf_kv_pool *pool);
+
 const char *aaf_kv_strerror(int status);
 
 #ifdef __cplusplus

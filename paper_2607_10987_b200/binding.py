@@ -106,6 +106,7 @@ SYMBOLS = {
     "aaf_kv_transfer_time_packed": (C.c_double, [C.c_double, C.c_double, C.c_double, C.c_double]),
     "aaf_kv_policy": (C.c_int, [C.c_int, C.c_double, C.c_double]),
     "aaf_kv_debug_expire_wait": (C.c_int, [_vp, C.c_uint64, _vp]),
+    "aaf_kv_debug_mark_unusable": (C.c_int, [_vp]),
     "aaf_kv_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -190,6 +191,7 @@ def aaf_kv_transfer_time_packed(kv_bytes, bandwidth, latency, pack_rate):
 def aaf_kv_policy(local_and_compatible, t_transfer, t_prefill):
     return _fn("aaf_kv_policy")(1 if local_and_compatible else 0, t_transfer, t_prefill)
 def aaf_kv_debug_expire_wait(pool, limit_cycles, stream): return _fn("aaf_kv_debug_expire_wait")(pool, limit_cycles, stream)
+def aaf_kv_debug_mark_unusable(pool): return _fn("aaf_kv_debug_mark_unusable")(pool)
 def aaf_kv_strerror(status): return _fn("aaf_kv_strerror")(status).decode()
 
 

@@ -1297,6 +1297,12 @@ int aaf_kv_debug_expire_wait(aaf_kv_pool *p, uint64_t limit_cycles, void *stream
     return launch_expire_wait(p->s, (long long)limit_cycles, p->meta_stream) == cudaSuccess ? AAF_OK : AAF_ERR_CUDA;
 }
 
+int aaf_kv_debug_mark_unusable(aaf_kv_pool *p) {
+    if (!p) return AAF_ERR_INVALID_ARG;
+    p->broken = true;
+    return AAF_OK;
+}
+
 int aaf_kv_set_timing(aaf_kv_pool *p, int enable) {
     if (!p) return AAF_ERR_INVALID_ARG;
     p->timing = enable != 0;

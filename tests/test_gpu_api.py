@@ -236,6 +236,30 @@ def test_calls_on_alternating_streams_do_not_overlap_their_copy_launches():
     assert gpu.o.sync_status() == 0
 
 
+def test_a_pool_marked_unusable_refuses_every_operator_and_changes_nothing():
+    """The documented exception to "an error changes nothing": after a CUDA failure inside an operator the pool
+    refuses all further work.  The state is entered here through the test hook, without any failure."""
+    gpu = GpuBackend(G, SEED)
+    o = gpu.o
+    buf = gpu.payload(SEED, 1, 40)
+    st, c = o.imp(buf, 40)
+    assert st == 0
+    before = gpu.snapshot()
+    assert binding.aaf_kv_debug_mark_unusable(o.h) == 0
+    out = torch.empty(40 * G.bpt, dtype=torch.uint8, device=o.device)
+    host = torch.empty(40 * G.bpt, dtype=torch.uint8).pin_memory()
+    E = binding.AAF_ERR_CUDA
+    assert o.materialize(c, 0, 40, out=out)[0] == E and o.imp(buf, 40)[0] == E and o.fork(c, 1)[0] == E
+    assert o.append([c], [40], [buf])[0] == E and o.compose([c, c])[0] == E and o.evict([c])[0] == E
+    assert o.compose_batch([[c], [c]])[0] == E and o.materialize_batch([c], [0], [40], [out]) == E
+    assert o.import_batch([buf], [40])[0] == E and o.append_host([c], [40], [host], out) == E
+    assert o.materialize_host(c, 0, 40, host, out) == E and o.import_host(host, 40, out)[0] == E
+    assert o.materialize_host_chunked(c, 0, 40, host, out, 16)[0] == E and o.import_host_chunked(host, 40, out, 16)[0] == E
+    assert o.evict_to_budget(0.0, 0.0, 1.0, 0)[0] == E
+    assert gpu.snapshot() == before and o.sync_status() == 0  # introspection still answers; nothing changed
+    o.close()
+
+
 def test_two_pools_of_different_geometry_interleaved():
     """Launch shapes and scratch are per pool: two pools with different rows, block sizes and engines,
     used alternately on the same stream, each stay bit-exact against their own oracle."""
