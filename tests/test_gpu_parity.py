@@ -78,8 +78,9 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
     outcomes = []
     for i in range(n_ops):
         live = cpu.o.live_ctxs()
-        kind = str(rng.choice(["import", "fork", "append", "compose", "evict", "materialize", "roundtrip", "budget"],
-                              p=[0.16, 0.12, 0.25, 0.14, 0.10, 0.13, 0.06, 0.04]))
+        kind = str(rng.choice(["import", "fork", "append", "compose", "evict", "materialize", "roundtrip", "budget",
+                               "compose_batch", "transfer_batch"],
+                              p=[0.15, 0.11, 0.22, 0.11, 0.10, 0.11, 0.05, 0.04, 0.06, 0.05]))
         if not live:
             kind = "import"
         pick = lambda: int(rng.choice(live)) if rng.random() > 0.04 else int(rng.integers(0, g.max_ctx))
@@ -101,6 +102,48 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
             segs = [pick() for _ in range(int(rng.integers(1, 4)))]
             fl = int(rng.integers(0, 2))
             res = [be.compose(segs, fl) for be in both]
+        elif kind in ("compose_batch", "transfer_batch"):
+            # Batched calls equal the oracle's loop of single calls when the loop succeeds throughout; when any
+            # call of the loop fails, the batch must fail as a whole and change nothing (the loop is tried on a copy).
+            import torch
+
+            before = cpu.snapshot()
+            trial = cpu.o.clone()
+            if kind == "compose_batch":
+                batch = [[pick() for _ in range(int(rng.integers(1, 4)))] for _ in range(int(rng.integers(1, 4)))]
+                fl = int(rng.integers(0, 2))
+                loop_ok = all(trial.compose(segs, fl)[0] == 0 for segs in batch)
+                st_g, r_g = gpu.o.compose_batch(batch, fl)
+                r_c = [cpu.compose(segs, fl)[1] for segs in batch] if loop_ok else None
+            else:
+                ranges = []
+                for _ in range(int(rng.integers(1, 4))):
+                    c = pick()
+                    T = cpu.o.ctx_len(c) or 4
+                    a = int(rng.integers(0, T))
+                    ranges.append((c, a, int(rng.integers(a, T + 1))))  # a == b -> INVALID_ARG
+                outs = [torch.empty(max(b - a, 1) * g.bpt, dtype=torch.uint8, device=gpu.o.device)
+                        for _, a, b in ranges]
+                bufs_c = [trial.materialize(c, a, b) for c, a, b in ranges]
+                loop_ok = all(st == 0 for st, _ in bufs_c) and \
+                    all(trial.imp(buf, b - a)[0] == 0 for (st, buf), (_, a, b) in zip(bufs_c, ranges))
+                st_g = gpu.o.materialize_batch([c for c, _, _ in ranges], [a for _, a, _ in ranges],
+                                               [b for _, _, b in ranges], outs)
+                r_g = None
+                if all(st == 0 for st, _ in bufs_c):  # the gathers alone are valid: compare them, then register
+                    assert st_g == 0, (i, kind, st_g)
+                    for (c, a, b), o_dev in zip(ranges, outs):
+                        assert np.array_equal(o_dev.cpu().numpy()[: (b - a) * g.bpt], cpu.materialize(c, a, b)[1])
+                    st_g, r_g = gpu.o.import_batch(outs, [b - a for _, a, b in ranges])
+                    r_c = [cpu.imp(buf, b - a)[1] for (_, buf), (_, a, b) in zip(bufs_c, ranges)] if loop_ok else None
+                else:
+                    assert st_g < 0, (i, kind)
+                    r_c = None
+            if loop_ok:
+                res = [(st_g, r_g), (0, r_c)]
+            else:
+                assert st_g < 0 and gpu.snapshot() == before, (i, kind, st_g)
+                res = [(st_g, None), (st_g, None)]
         elif kind == "evict":
             who = [pick() for _ in range(int(rng.integers(1, 3)))]
             res = [be.evict(who) for be in both]
