@@ -112,7 +112,9 @@ def random_walk(g: Geometry, seed: int, n_ops: int, engine: int):
             if kind == "compose_batch":
                 batch = [[pick() for _ in range(int(rng.integers(1, 4)))] for _ in range(int(rng.integers(1, 4)))]
                 fl = int(rng.integers(0, 2))
-                loop_ok = all(trial.compose(segs, fl)[0] == 0 for segs in batch)
+                # (a result of the same batch cannot be a segment: every segment must be live before the call)
+                loop_ok = all(c in live for segs in batch for c in segs) and \
+                    all(trial.compose(segs, fl)[0] == 0 for segs in batch)
                 st_g, r_g = gpu.o.compose_batch(batch, fl)
                 r_c = [cpu.compose(segs, fl)[1] for segs in batch] if loop_ok else None
             else:
