@@ -547,11 +547,40 @@ def extra_report(args):
         def floor():
             one.add_(1.0)
 
+        def breakdown(fn, wait):
+            """one call at a time: time inside the call (host side: validation, launch, bookkeeping, binding) and
+            time until the device has finished it"""
+            host, total = [], []
+            for _ in range(300):
+                wait()
+                t0 = time.perf_counter_ns()
+                fn()
+                t1 = time.perf_counter_ns()
+                wait()
+                t2 = time.perf_counter_ns()
+                host.append(t1 - t0); total.append(t2 - t0)
+            host.sort(); total.sort()
+            return {"host_call_us_median": host[len(host) // 2] / 1e3, "call_plus_wait_us_median": total[len(total) // 2] / 1e3}
+
+        kid = []
+
+        def fork1():
+            kid[:] = be.fork(root, 1)[1]
+
+        def evict1():
+            be.evict(kid)
+
+        def fork_then_evict():  # keeps the handle count constant across iterations
+            fork1(); evict1()
+
         out.update({"context_blocks": T // 16,
                     "fork16_then_evict16 (8192 + 8192 entries)": rate(fork_evict, 2),
                     "fork1_then_evict1 (512 + 512 entries)": rate(fork1_evict, 2),
                     "table_only_compose_then_evict (1024 entries)": rate(compose_evict, 2),
-                    "launch_floor_trivial_torch_kernel": rate(floor, 1)})
+                    "launch_floor_trivial_torch_kernel": rate(floor, 1),
+                    "one_call_at_a_time": {
+                        "fork1_plus_evict1 (two calls)": breakdown(fork_then_evict, torch.cuda.synchronize),
+                        "trivial_torch_kernel": breakdown(floor, torch.cuda.synchronize)}})
     elif args.workload == "transfer":
         # pack / unpack against host memory: one shot versus chunked with per-chunk completion flags
         g, seed, T = configs.LLAMA8B, configs.SEED_BASE + 2, 8187
