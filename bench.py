@@ -731,8 +731,14 @@ def measure_step(w, args, cl, dev_index, steps, warmup, min_seconds, clocks_for_
     free_b, _total = torch.cuda.mem_get_info(dev)
     n_blocks = g.n_blocks
     need = lambda nb: g.n_layers * nb * 2 * g.run + 4 * T * g.bpt + (8 << 30)
-    while need(n_blocks) > free_b and n_blocks > 4096:
+    # blocks one step holds at its peak: sender's and receiver's context, every agent's continuation and COW block,
+    # the merged pair
+    step_blocks = 2 * g.nblk(T) + agents * (g.nblk(T + n_new) - g.nblk(T) + 1) + g.nblk(2 * (T + n_new)) + 64
+    while need(n_blocks) > free_b and n_blocks // 2 >= step_blocks:
         n_blocks //= 2  # recorded in config.n_blocks when the device lacks memory for the full pool
+    if need(n_blocks) > free_b:
+        raise RuntimeError(f"{w['name']}: needs {need(n_blocks) / 2**30:.0f} GiB of device memory, "
+                           f"{free_b / 2**30:.0f} GiB are free")
     pool = KVPool(g.n_layers, g.n_kv_heads, g.head_dim, g.block_size, g.elt_bytes, n_blocks, g.max_ctx,
                   g.max_blocks_per_ctx, free_order=configs.free_order(seed, n_blocks), device=dev_index)
     pool.set_copy_engine(args.engine)
@@ -907,21 +913,28 @@ def main():
     if args.workload == "8b" and not args.no_extra:
         single = Cluster(torch, dist, dev, 1, backend)  # replicas do not wait for each other here
         pw = {}
-        w70 = workload("70b")
-        r70 = measure_step(w70, args, single, dev_index, max(3, min(args.steps, 10)), 3, args.min_seconds, False, False)
-        rec = kernel_record(r70["moved_per_step"] * max(3, min(args.steps, 10)) * r70["repeats"], r70["copy_ms"],
-                            r70["copy_launches"], peak)
-        rec.update({"workload": r70["name"], "whole_step_GBps": r70["value_per_replica"], "ms_per_step": r70["ms_per_step"],
-                    "repeats": r70["repeats"], "pool_GiB": r70["pool_GiB"], "per_class_GBps": r70["per_class"]})
-        pw["70b"] = rec
         k = max(3, min(args.steps, 10))
-        for name, lv in compose_levels(args, peak, k, 2, copy_all=False).items():
-            pw["compose_" + name] = lv
-        pw["cow"] = cow_stress(args, peak, k, 2)
-        pw["cow_70b"] = cow_stress(args, peak, k, 2, n_layers=80)
-        for name, rec in suffix_transfers(args, peak, k, 2).items():
-            if isinstance(rec, dict):
-                pw["suffix_" + name] = rec
+
+        def step70():
+            r70 = measure_step(workload("70b"), args, single, dev_index, k, 3, args.min_seconds, False, False)
+            rec = kernel_record(r70["moved_per_step"] * k * r70["repeats"], r70["copy_ms"], r70["copy_launches"], peak)
+            rec.update({"workload": r70["name"], "whole_step_GBps": r70["value_per_replica"],
+                        "ms_per_step": r70["ms_per_step"], "repeats": r70["repeats"], "pool_GiB": r70["pool_GiB"],
+                        "per_class_GBps": r70["per_class"]})
+            return {"70b": rec}
+
+        parts = (step70,
+                 lambda: {"compose_" + n: lv for n, lv in compose_levels(args, peak, k, 2, copy_all=False).items()},
+                 lambda: {"cow": cow_stress(args, peak, k, 2)},
+                 lambda: {"cow_70b": cow_stress(args, peak, k, 2, n_layers=80)},
+                 lambda: {"suffix_" + n: rec for n, rec in suffix_transfers(args, peak, k, 2).items()
+                          if isinstance(rec, dict)})
+        for part in parts:  # a sub-workload that cannot run here (device memory) must not cost the headline line
+            try:
+                pw.update(part())
+            except (RuntimeError, AssertionError) as exc:
+                pw.setdefault("skipped", []).append(f"{type(exc).__name__}: {str(exc)[:200]}")
+                torch.cuda.empty_cache()
         roofline["per_workload"] = pw
 
     if rank != 0:
