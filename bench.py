@@ -289,6 +289,18 @@ def cow_stress(args, peak, steps, warmup, n_layers=32):
             acc["append_ms"] += dms["append"]; acc["append_bytes"] += b; acc["launches"] += dl["append"]
             acc["fork_ms"] += ms_f; acc["evict_ms"] += ms_e
     assert be.o.sync_status() == 0 and be.o.stats()["cow_count"] == kids_n * (warmup + steps)
+    # the same at the fan-out of the workload configs (16 agents at the 8B shape, 8 at the 70B shape): a copy of a
+    # few tens of MiB, i.e. a latency figure: kernel time and time of the whole call on an idle stream
+    few = 16 if n_layers <= 32 else 8
+    lat = {"kernel_ms": 0.0, "call_ms": 0.0}
+    for it in range(warmup + steps):
+        st, root = be.imp(root_buf, T)
+        st, kids = be.fork(root, few)
+        ms_a, dms, dl, b = timed_ops(be.o, lambda: be.append(kids, [1] * few, one[:few]))
+        be.evict(kids + [root])
+        if it >= warmup:
+            lat["kernel_ms"] += dms["append"] / steps; lat["call_ms"] += ms_a / steps
+    lat.update({"agents": few, "bytes_copied_MiB": b / 2**20})
     rec = kernel_record(2 * acc["append_bytes"], acc["append_ms"], acc["launches"], peak)
     written = acc["append_bytes"] / (acc["append_ms"] * 1e-3) / 1e9
     # the counted rate (read + written) exceeds the DRAM peak because the reads are L2 hits: the figure to hold
@@ -298,7 +310,8 @@ def cow_stress(args, peak, steps, warmup, n_layers=32):
                 "traffic_source": "modelled: the bytes written (the 11 shared source rows are read from the L2)",
                 "note": "achieved = bytes written per second (DRAM side); the 1024 children read the same 11 rows",
                 "children": kids_n, "rows_copied_per_child": T % g.block_size, "n_layers": n_layers,
-                "fork_1024_ms": acc["fork_ms"] / steps, "evict_1024_plus_1_ctx_ms": acc["evict_ms"] / steps})
+                "fork_1024_ms": acc["fork_ms"] / steps, "evict_1024_plus_1_ctx_ms": acc["evict_ms"] / steps,
+                "first_append_of_the_config_fanout": lat})
     del be
     return rec
 
